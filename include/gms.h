@@ -1,0 +1,234 @@
+/*
+ * gms.h -- C ABI of the restore / digest / verify data path of a GPU Memory
+ * Service (GMS), written for NVIDIA B200 (sm_100a).
+ *
+ * Background (paper: "Fast Recovery for LLM Serving via Decoupled Device
+ * Memory Lifetime in Dynamo").  Section 3.2 moves model state into device
+ * allocations owned by a per-GPU service so that it outlives an engine:
+ * a writer populates the allocations and commits them, later engines attach
+ * read-only.  Section 4 (GMS paragraph) adds that the client "records tensor
+ * layouts" before commit and that, when the service is cold, a separate
+ * read-write client repopulates model state in parallel with process restore.
+ * Section 3.1 models the cost of that as S / B_eff, and Section 5.2 observes
+ * that today's tool copies device memory serially and leaves the link idle.
+ * Section 2.2 allows reuse of surviving allocations only if their contents are
+ * intact.  The paper leaves the bulk data path and the integrity check
+ * unspecified; this library is that path:
+ *
+ *   gms_manifest_build   the recorded tensor layout, turned into a work list
+ *   gms_restore          scatter a packed snapshot image into the allocations,
+ *                        digesting every 4 KiB block in the same pass
+ *   gms_digest           digest surviving allocations in place (no writes)
+ *   gms_verify           compare digests with the ones recorded at commit and
+ *                        name the blocks that differ
+ *   gms_kv_restore       scatter a subset of paged KV blocks (Section 6,
+ *                        "Preserving KV state") through a block-index list
+ *
+ * The digest (fixed by this library, not by the paper; all arithmetic on
+ * uint64_t, wrapping):
+ *   mix(z):  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9;
+ *            z = (z ^ (z >> 27)) * 0x94D049BB133111EB;  return z ^ (z >> 31);
+ *   block digest  D   = XOR_{i<512} mix(w_i ^ i*G), G = 0x9E3779B97F4A7C15,
+ *            w_i the little-endian u64 words of the block, a block shorter
+ *            than 4096 bytes being extended with zero bytes;
+ *   tensor digest T   = XOR_{b<nb} mix(D_b ^ b*G), blocks cut relative to the
+ *            tensor's first byte, nb = ceil(nbytes / 4096); nbytes = 0: T = 0.
+ * Results are exact integers; every output of this library is bit-reproducible.
+ *
+ * Conventions.
+ *  - Every function returns int: GMS_OK (0) or a negative GMS_ERR_* value.
+ *    Nothing throws, aborts or traps.  Host-detectable errors are returned
+ *    before any device work is enqueued.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  Device work is asynchronous with respect to the host; outputs
+ *    are valid once the stream has been synchronised.
+ *  - Pointers are marked (device), (host) or (device-accessible).  The caller
+ *    owns every buffer it passes and keeps it alive until the stream work has
+ *    completed.  The library allocates only the manifest's own small tables
+ *    (32 bytes per <=128 KiB of payload, plus the recorded digests).
+ *  - Calls that use the same manifest must not overlap on the GPU (they share
+ *    the manifest's work counter and status word); enqueue them on one stream
+ *    or order them with events.
+ */
+#ifndef GMS_H
+#define GMS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GMS_BLOCK_BYTES 4096u
+
+/* status codes */
+#define GMS_OK 0
+#define GMS_ERR_NULL (-1)     /* a required pointer is NULL                                   */
+#define GMS_ERR_ALIGN (-2)    /* src_offset or dst not 16-byte aligned; bad block_bytes       */
+#define GMS_ERR_RANGE (-3)    /* src_offset + nbytes exceeds the image, or overflows          */
+#define GMS_ERR_OVERLAP (-4)  /* two destination ranges intersect                             */
+#define GMS_ERR_DUP_ID (-5)   /* two entries carry the same tensor_id                         */
+#define GMS_ERR_NOMEM (-6)    /* host or device allocation of the manifest's tables failed    */
+#define GMS_ERR_CUDA (-7)     /* a CUDA runtime call failed; text via gms_last_cuda_error()   */
+#define GMS_ERR_KIND (-8)     /* image_kind is not one of GMS_SRC_*                           */
+#define GMS_ERR_TIMEOUT (-9)  /* a bounded device-side wait gave up (see device status word)  */
+#define GMS_ERR_STATE (-10)   /* manifest has no device tables / no recorded digests          */
+#define GMS_ERR_ARG (-11)     /* an argument is out of its documented range                   */
+
+/* where the packed snapshot image lives */
+#define GMS_SRC_DEVICE 0u      /* device memory (a staging buffer in HBM)                     */
+#define GMS_SRC_HOST_MAPPED 1u /* pinned host memory mapped into the device address space     */
+
+/* gms_manifest_build flags */
+#define GMS_BUILD_HOST_ONLY 1u /* validate and build the work list on the host only (no CUDA
+                                  call is made; device entry points return GMS_ERR_STATE)     */
+
+/* bits of the device status word */
+#define GMS_DEV_TIMEOUT 1ull   /* a warp gave up waiting for one of its own bulk copies       */
+
+typedef struct gms_manifest gms_manifest; /* opaque */
+
+/* One recorded tensor layout (Section 4: "the client records tensor layouts"). */
+typedef struct {
+    uint64_t tensor_id;  /* caller's identifier, unique within a manifest                     */
+    uint64_t src_offset; /* byte offset of the tensor in the packed image, 16-byte aligned    */
+    void *dst;           /* (device) destination, 16-byte aligned                             */
+    uint64_t nbytes;     /* length in bytes, any value >= 0                                   */
+} gms_entry;
+
+typedef struct {
+    uint64_t tensor_id; /* as given in the entry                                              */
+    uint64_t block;     /* 4 KiB block index relative to the tensor's first byte              */
+} gms_mismatch;
+
+/*
+ * gms_manifest_build -- Section 4, GMS paragraph (layout record made before
+ * commit); Section 3.2 (the allocations it describes).
+ * Validates `entries` (host, n of them) against an image of `image_bytes`
+ * bytes and builds the work list that gms_restore / gms_digest walk: every
+ * tensor is cut into chunks of at most 32 blocks so that thousands of small
+ * and a few huge tensors are served by one persistent launch.
+ * Block digests are laid out in entry order: tensor t owns slots
+ * [first_block(t), first_block(t) + ceil(nbytes_t/4096)).
+ * Errors: NULL, ALIGN, RANGE, OVERLAP (destinations; overlapping sources are
+ * legal), DUP_ID, NOMEM, CUDA.  nbytes == 0 is legal (no blocks, T = 0).
+ * Bytes of a destination beyond nbytes are never written.
+ * On success *out owns host and (unless GMS_BUILD_HOST_ONLY) device tables on
+ * the current device; release it with gms_manifest_destroy.
+ */
+int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes, uint32_t flags, gms_manifest **out);
+int gms_manifest_destroy(gms_manifest *m);
+
+/* Sizes of the outputs: number of entries, of digest blocks, and of payload bytes. */
+int gms_manifest_info(const gms_manifest *m, uint64_t *n_tensors, uint64_t *n_blocks, uint64_t *payload_bytes);
+/* First digest-block slot of entry `entry_index`. */
+int gms_manifest_block_base(const gms_manifest *m, size_t entry_index, uint64_t *first_block);
+/* Work-list introspection (host): number of chunks, and chunk `i` as
+ * (entry index, byte offset inside the tensor, bytes).  Chunks partition every tensor. */
+int gms_manifest_chunk_count(const gms_manifest *m, uint64_t *n_chunks);
+int gms_manifest_chunk(const gms_manifest *m, uint64_t i, uint64_t *entry_index, uint64_t *tensor_byte_offset,
+                       uint64_t *nbytes);
+
+/*
+ * gms_manifest_set_expected -- Section 3.2: commit makes the model state
+ * immutable; the digests recorded at that moment are what later reuse is
+ * checked against.  Copies n_blocks block digests (device) into the manifest
+ * (device-to-device, on `stream`).
+ */
+int gms_manifest_set_expected(gms_manifest *m, const uint64_t *d_block_digests, void *stream);
+
+/*
+ * gms_restore -- Section 4 (cold-service repopulation), Section 3.3
+ * (reconstruction after a device-invalidating failure), cost model S/B_eff of
+ * Section 3.1.  For every entry: dst[0, nbytes) <- image[src_offset, +nbytes),
+ * and, in the same pass over the bytes, D for each block and T for each tensor.
+ *   image            (device-accessible) start of the packed image:
+ *                    device memory for GMS_SRC_DEVICE, the device-side
+ *                    address of pinned mapped host memory for
+ *                    GMS_SRC_HOST_MAPPED; 16-byte aligned
+ *   d_block_digests  (device) n_blocks u64, may be NULL
+ *   d_tensor_digests (device) n u64, may be NULL
+ * One persistent kernel (plus a one-block prologue that clears accumulators);
+ * no per-tensor launches.  Errors: NULL, ALIGN, KIND, STATE, CUDA.
+ */
+int gms_restore(const gms_manifest *m, const void *image, uint32_t image_kind, uint64_t *d_block_digests,
+                uint64_t *d_tensor_digests, void *stream);
+
+/*
+ * gms_digest -- Section 3.2 (a replacement engine attaches surviving
+ * allocations read-only) and Section 2.2 (reuse only if contents are intact).
+ * Same outputs as gms_restore, computed over the destinations where they lie;
+ * the destinations are only read.
+ */
+int gms_digest(const gms_manifest *m, uint64_t *d_block_digests, uint64_t *d_tensor_digests, void *stream);
+
+/*
+ * gms_verify -- the trust decision of Section 2.2.  Compares
+ * d_block_digests[n_blocks] (device) with the digests recorded by
+ * gms_manifest_set_expected and writes the differing (tensor_id, block) pairs
+ * to d_out (device, `cap` slots) in ascending (entry position, block) order.
+ * *d_count (device, u64) receives the total number of differing blocks, which
+ * may exceed cap; only min(count, cap) slots of d_out are written.
+ * Errors: NULL, STATE (nothing recorded), CUDA.
+ */
+int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_mismatch *d_out, uint32_t cap,
+               uint64_t *d_count, void *stream);
+
+/* Device status word of the manifest's last call (synchronises `stream`). 0 = clean. */
+int gms_last_device_status(const gms_manifest *m, void *stream, uint64_t *word);
+
+/* A paged KV pool: n_planes planes (layer x {K,V}) of n_blocks blocks. */
+typedef struct {
+    void *base;            /* (device) 16-byte aligned                                        */
+    uint64_t plane_stride; /* bytes between planes, multiple of 16                            */
+    uint64_t block_stride; /* bytes between blocks of a plane, multiple of 16, >= block_bytes */
+    uint32_t n_planes;
+    uint32_t n_blocks;
+    uint32_t block_bytes;  /* multiple of 4096, at most 131072                                */
+    uint32_t reserved;     /* 0                                                               */
+} gms_kv_pool;
+
+/*
+ * gms_kv_restore -- Section 6, "Preserving KV state": committed KV blocks
+ * kept in host memory or storage are put back after recovery.  For j < n_sel
+ * and every plane p:
+ *   pool[p][d_block_ids[j]] <- image + p*img_plane_stride + j*img_slot_stride
+ * (block_bytes bytes each), with digests
+ *   d_block_digests[(j*n_planes + p)*k + c]  for 4 KiB block c of that copy,
+ *                                            k = block_bytes/4096;
+ *   d_kv_digests[j] = XOR_q mix(D_q ^ q*G), q = p*k + c  (the tensor digest of
+ *                                            the slot's planes concatenated).
+ * An id outside [0, n_blocks) is skipped: nothing is written to the pool, its
+ * digests are 0, and d_status[0] counts it.  d_status[1] receives the device
+ * status word.  Ids must be distinct (the caller's duty; duplicates race).
+ *   image        (device-accessible) as for gms_restore; strides multiples of 16
+ *   d_block_ids  (device) int32[n_sel]
+ *   d_block_digests (device) n_sel*n_planes*k u64, may be NULL
+ *   d_kv_digests (device) n_sel u64, may be NULL
+ *   d_status     (device) 2 u64
+ * Errors: NULL, ALIGN, KIND, ARG, CUDA.
+ */
+int gms_kv_restore(const gms_kv_pool *pool, const void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
+                   uint32_t image_kind, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
+                   uint64_t *d_kv_digests, uint64_t *d_status, void *stream);
+
+/*
+ * Pinned, device-mapped host memory for a GMS_SRC_HOST_MAPPED image (the
+ * host-resident snapshot of Section 3.1 step 3 / Section 6).  *device_view is
+ * the address to pass as `image`.
+ */
+int gms_host_image_alloc(uint64_t nbytes, void **host_ptr, void **device_view);
+int gms_host_image_free(void *host_ptr);
+
+/* Launch geometry of the streaming kernels on the current device (for reporting). */
+int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *smem_bytes);
+
+const char *gms_strerror(int status);
+const char *gms_last_cuda_error(void); /* text of the last failed CUDA call on this thread */
+uint32_t gms_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GMS_H */

@@ -1,0 +1,440 @@
+// Host side of the C ABI declared in include/gms.h: validation of the layout
+// record, construction of the persistent kernels' work list, and the entry
+// points that enqueue the kernels.  There is no CPU implementation of the data
+// path here: every entry point either launches the CUDA kernels or fails.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <numeric>
+#include <string>
+#include <vector>
+
+#include "../../include/gms.h"
+#include "gms_internal.h"
+
+using gms::Chunk;
+
+struct gms_manifest {
+    std::vector<gms_entry> entries;
+    std::vector<uint64_t> block_base;  // n + 1 prefix sums of per-tensor block counts
+    std::vector<Chunk> chunks;
+    uint64_t image_bytes = 0, payload = 0, n_blocks = 0;
+    bool host_only = false;
+    int device = -1;
+    // device tables (one allocation) and the recorded digests (allocated on first use)
+    uint8_t *d_tables = nullptr;
+    Chunk *d_chunks = nullptr;
+    uint64_t *d_block_base = nullptr, *d_tensor_ids = nullptr, *d_seg_offset = nullptr;
+    uint32_t *d_seg_count = nullptr;
+    unsigned int *d_counter = nullptr;
+    unsigned long long *d_status = nullptr;
+    uint64_t *d_expected = nullptr;
+    bool has_expected = false;
+    uint32_t n_segments = 0;
+};
+
+namespace {
+
+thread_local std::string t_cuda_error;
+
+int cuda_fail(cudaError_t e)
+{
+    t_cuda_error = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e);
+    (void)cudaGetLastError();  // clear the sticky-less error state
+    return GMS_ERR_CUDA;
+}
+#define GMS_CUDA(call)                         \
+    do {                                       \
+        cudaError_t e_ = (call);               \
+        if (e_ != cudaSuccess) return cuda_fail(e_); \
+    } while (0)
+
+uint64_t blocks_of(uint64_t nbytes) { return nbytes / gms::kBlockBytes + (nbytes % gms::kBlockBytes ? 1 : 0); }
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Cut every tensor into runs of at most `chunk_blocks` digest blocks.  Large runs first, so that
+// the dynamic claim order ends on the small ones and the last wave of warps finishes together.
+void build_chunks(gms_manifest &m, uint32_t chunk_blocks)
+{
+    const uint64_t chunk_bytes = (uint64_t)chunk_blocks * gms::kBlockBytes;
+    m.chunks.clear();
+    for (size_t t = 0; t < m.entries.size(); ++t) {
+        const gms_entry &e = m.entries[t];
+        for (uint64_t off = 0; off < e.nbytes; off += chunk_bytes) {
+            Chunk c;
+            c.src_off = e.src_offset + off;
+            c.dst = reinterpret_cast<uint64_t>(e.dst) + off;
+            c.nbytes = (uint32_t)std::min<uint64_t>(chunk_bytes, e.nbytes - off);
+            c.tensor = (uint32_t)t;
+            c.gblock0 = (uint32_t)(m.block_base[t] + off / gms::kBlockBytes);
+            c.tblock0 = (uint32_t)(off / gms::kBlockBytes);
+            m.chunks.push_back(c);
+        }
+    }
+    std::stable_sort(m.chunks.begin(), m.chunks.end(), [](const Chunk &a, const Chunk &b) { return a.nbytes > b.nbytes; });
+}
+
+int check_kind(const void *image, uint32_t kind)
+{
+    if (kind != GMS_SRC_DEVICE && kind != GMS_SRC_HOST_MAPPED) return GMS_ERR_KIND;
+    cudaPointerAttributes at;
+    cudaError_t e = cudaPointerGetAttributes(&at, image);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (kind == GMS_SRC_DEVICE && at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged) return GMS_ERR_KIND;
+    if (kind == GMS_SRC_HOST_MAPPED && at.type != cudaMemoryTypeHost) return GMS_ERR_KIND;
+    return GMS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes, uint32_t flags, gms_manifest **out)
+{
+    if (!out || (n && !entries)) return GMS_ERR_NULL;
+    *out = nullptr;
+    if (flags & ~GMS_BUILD_HOST_ONLY) return GMS_ERR_ARG;
+    if (n >= 0xffffffffull) return GMS_ERR_RANGE;
+
+    // ---- validation (all on the host, before any CUDA call)
+    uint64_t n_blocks = 0, payload = 0;
+    for (size_t t = 0; t < n; ++t) {
+        const gms_entry &e = entries[t];
+        if ((e.src_offset & 15u) || (reinterpret_cast<uint64_t>(e.dst) & 15u)) return GMS_ERR_ALIGN;
+        if (e.nbytes && !e.dst) return GMS_ERR_NULL;
+        if (e.src_offset > image_bytes || e.nbytes > image_bytes - e.src_offset) return GMS_ERR_RANGE;
+        if (reinterpret_cast<uint64_t>(e.dst) + e.nbytes < reinterpret_cast<uint64_t>(e.dst)) return GMS_ERR_RANGE;
+        n_blocks += blocks_of(e.nbytes);
+        payload += e.nbytes;
+        if (n_blocks >= 0xffffffffull) return GMS_ERR_RANGE;  // digest slots are indexed with 32 bits on the device
+    }
+    try {
+        std::vector<uint32_t> order(n);
+        std::iota(order.begin(), order.end(), 0u);
+        std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return entries[a].tensor_id < entries[b].tensor_id; });
+        for (size_t i = 1; i < n; ++i)
+            if (entries[order[i]].tensor_id == entries[order[i - 1]].tensor_id) return GMS_ERR_DUP_ID;
+        // destinations pairwise disjoint: sort the non-empty ones by address, compare neighbours
+        std::vector<uint32_t> live;
+        for (uint32_t t = 0; t < n; ++t)
+            if (entries[t].nbytes) live.push_back(t);
+        std::sort(live.begin(), live.end(), [&](uint32_t a, uint32_t b) {
+            return reinterpret_cast<uint64_t>(entries[a].dst) < reinterpret_cast<uint64_t>(entries[b].dst);
+        });
+        for (size_t i = 1; i < live.size(); ++i) {
+            const gms_entry &p = entries[live[i - 1]], &q = entries[live[i]];
+            if (reinterpret_cast<uint64_t>(p.dst) + p.nbytes > reinterpret_cast<uint64_t>(q.dst)) return GMS_ERR_OVERLAP;
+        }
+
+        gms_manifest *m = new gms_manifest();
+        m->entries.assign(entries, entries + n);
+        m->image_bytes = image_bytes;
+        m->payload = payload;
+        m->n_blocks = n_blocks;
+        m->host_only = (flags & GMS_BUILD_HOST_ONLY) != 0;
+        m->block_base.resize(n + 1);
+        uint64_t acc = 0;
+        for (size_t t = 0; t < n; ++t) {
+            m->block_base[t] = acc;
+            acc += blocks_of(entries[t].nbytes);
+        }
+        m->block_base[n] = acc;
+
+        // ---- chunk size: small enough that every warp of the grid gets several chunks
+        uint32_t total_warps = 148 * 12;
+        if (!m->host_only) {
+            gms::Geometry g;
+            cudaError_t e = gms::get_geometry(&g);
+            if (e != cudaSuccess) {
+                delete m;
+                return cuda_fail(e);
+            }
+            total_warps = g.grid * g.warps;
+            (void)cudaGetDevice(&m->device);
+        }
+        uint32_t max_chunk = 16;
+        if (const char *v = getenv("GMS_CHUNK_BLOCKS")) {
+            const long x = atol(v);
+            if (x >= 1 && x <= (long)gms::kMaxChunkBlocks) max_chunk = (uint32_t)x;
+        }
+        const uint64_t want = n_blocks / (8ull * total_warps);
+        const uint32_t chunk_blocks = (uint32_t)std::min<uint64_t>(max_chunk, std::max<uint64_t>(1, want));
+        build_chunks(*m, chunk_blocks);
+        m->n_segments = (uint32_t)((n_blocks + gms::kVerifySegBlocks - 1) / gms::kVerifySegBlocks);
+
+        // ---- device tables
+        if (!m->host_only) {
+            const size_t o_chunks = 0;
+            const size_t o_base = align_up(o_chunks + m->chunks.size() * sizeof(Chunk), 256);
+            const size_t o_ids = align_up(o_base + (n + 1) * sizeof(uint64_t), 256);
+            const size_t o_segoff = align_up(o_ids + n * sizeof(uint64_t), 256);
+            const size_t o_segcnt = align_up(o_segoff + (size_t)m->n_segments * sizeof(uint64_t), 256);
+            const size_t o_ctr = align_up(o_segcnt + (size_t)m->n_segments * sizeof(uint32_t), 256);
+            const size_t o_status = o_ctr + 128;
+            const size_t total = o_status + 128;
+            std::vector<uint8_t> h(total, 0);
+            if (!m->chunks.empty()) memcpy(h.data() + o_chunks, m->chunks.data(), m->chunks.size() * sizeof(Chunk));
+            memcpy(h.data() + o_base, m->block_base.data(), (n + 1) * sizeof(uint64_t));
+            for (size_t t = 0; t < n; ++t) memcpy(h.data() + o_ids + t * 8, &entries[t].tensor_id, 8);
+            cudaError_t e = cudaMalloc(&m->d_tables, total);
+            if (e != cudaSuccess) {
+                delete m;
+                (void)cudaGetLastError();
+                return e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : cuda_fail(e);
+            }
+            e = cudaMemcpy(m->d_tables, h.data(), total, cudaMemcpyHostToDevice);
+            if (e != cudaSuccess) {
+                cudaFree(m->d_tables);
+                delete m;
+                return cuda_fail(e);
+            }
+            m->d_chunks = reinterpret_cast<Chunk *>(m->d_tables + o_chunks);
+            m->d_block_base = reinterpret_cast<uint64_t *>(m->d_tables + o_base);
+            m->d_tensor_ids = reinterpret_cast<uint64_t *>(m->d_tables + o_ids);
+            m->d_seg_offset = reinterpret_cast<uint64_t *>(m->d_tables + o_segoff);
+            m->d_seg_count = reinterpret_cast<uint32_t *>(m->d_tables + o_segcnt);
+            m->d_counter = reinterpret_cast<unsigned int *>(m->d_tables + o_ctr);
+            m->d_status = reinterpret_cast<unsigned long long *>(m->d_tables + o_status);
+        }
+        *out = m;
+        return GMS_OK;
+    } catch (const std::bad_alloc &) {
+        return GMS_ERR_NOMEM;
+    }
+}
+
+int gms_manifest_destroy(gms_manifest *m)
+{
+    if (!m) return GMS_OK;
+    int rc = GMS_OK;
+    if (m->d_expected && cudaFree(m->d_expected) != cudaSuccess) rc = GMS_ERR_CUDA;
+    if (m->d_tables && cudaFree(m->d_tables) != cudaSuccess) rc = GMS_ERR_CUDA;
+    delete m;
+    return rc;
+}
+
+int gms_manifest_info(const gms_manifest *m, uint64_t *n_tensors, uint64_t *n_blocks, uint64_t *payload_bytes)
+{
+    if (!m) return GMS_ERR_NULL;
+    if (n_tensors) *n_tensors = m->entries.size();
+    if (n_blocks) *n_blocks = m->n_blocks;
+    if (payload_bytes) *payload_bytes = m->payload;
+    return GMS_OK;
+}
+
+int gms_manifest_block_base(const gms_manifest *m, size_t entry_index, uint64_t *first_block)
+{
+    if (!m || !first_block) return GMS_ERR_NULL;
+    if (entry_index >= m->entries.size()) return GMS_ERR_ARG;
+    *first_block = m->block_base[entry_index];
+    return GMS_OK;
+}
+
+int gms_manifest_chunk_count(const gms_manifest *m, uint64_t *n_chunks)
+{
+    if (!m || !n_chunks) return GMS_ERR_NULL;
+    *n_chunks = m->chunks.size();
+    return GMS_OK;
+}
+
+int gms_manifest_chunk(const gms_manifest *m, uint64_t i, uint64_t *entry_index, uint64_t *tensor_byte_offset, uint64_t *nbytes)
+{
+    if (!m) return GMS_ERR_NULL;
+    if (i >= m->chunks.size()) return GMS_ERR_ARG;
+    const Chunk &c = m->chunks[i];
+    if (entry_index) *entry_index = c.tensor;
+    if (tensor_byte_offset) *tensor_byte_offset = (uint64_t)c.tblock0 * gms::kBlockBytes;
+    if (nbytes) *nbytes = c.nbytes;
+    return GMS_OK;
+}
+
+int gms_manifest_set_expected(gms_manifest *m, const uint64_t *d_block_digests, void *stream)
+{
+    if (!m || (m->n_blocks && !d_block_digests)) return GMS_ERR_NULL;
+    if (m->host_only) return GMS_ERR_STATE;
+    if (!m->d_expected && m->n_blocks) {
+        cudaError_t e = cudaMalloc(&m->d_expected, m->n_blocks * sizeof(uint64_t));
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            return e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : cuda_fail(e);
+        }
+    }
+    GMS_CUDA(gms::launch_copy_u64(m->d_expected, d_block_digests, m->n_blocks, static_cast<cudaStream_t>(stream)));
+    m->has_expected = true;
+    return GMS_OK;
+}
+
+static int stream_call(const gms_manifest *m, const void *image, bool store, uint64_t *d_block_digests,
+                       uint64_t *d_tensor_digests, void *stream)
+{
+    gms::StreamArgs a;
+    a.chunks = m->d_chunks;
+    a.n_chunks = (uint32_t)m->chunks.size();
+    a.image = static_cast<const uint8_t *>(image);
+    a.block_digests = d_block_digests;
+    a.tensor_digests = d_tensor_digests;
+    a.n_tensors = (uint32_t)m->entries.size();
+    a.work_counter = m->d_counter;
+    a.status = m->d_status;
+    GMS_CUDA(store ? gms::launch_restore(a, static_cast<cudaStream_t>(stream))
+                   : gms::launch_digest(a, static_cast<cudaStream_t>(stream)));
+    return GMS_OK;
+}
+
+int gms_restore(const gms_manifest *m, const void *image, uint32_t image_kind, uint64_t *d_block_digests,
+                uint64_t *d_tensor_digests, void *stream)
+{
+    if (!m || (!image && m->payload)) return GMS_ERR_NULL;
+    if (image_kind != GMS_SRC_DEVICE && image_kind != GMS_SRC_HOST_MAPPED) return GMS_ERR_KIND;
+    if (reinterpret_cast<uint64_t>(image) & 15u) return GMS_ERR_ALIGN;
+    if (m->host_only) return GMS_ERR_STATE;
+    if (image) {
+        const int rc = check_kind(image, image_kind);
+        if (rc) return rc;
+    }
+    return stream_call(m, image, true, d_block_digests, d_tensor_digests, stream);
+}
+
+int gms_digest(const gms_manifest *m, uint64_t *d_block_digests, uint64_t *d_tensor_digests, void *stream)
+{
+    if (!m) return GMS_ERR_NULL;
+    if (m->host_only) return GMS_ERR_STATE;
+    return stream_call(m, nullptr, false, d_block_digests, d_tensor_digests, stream);
+}
+
+int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_mismatch *d_out, uint32_t cap, uint64_t *d_count,
+               void *stream)
+{
+    if (!m || !d_count || (cap && !d_out) || (m->n_blocks && !d_block_digests)) return GMS_ERR_NULL;
+    if (m->host_only || !m->has_expected) return GMS_ERR_STATE;
+    gms::VerifyArgs a;
+    a.computed = d_block_digests;
+    a.expected = m->d_expected;
+    a.n_blocks = m->n_blocks;
+    a.block_base = m->d_block_base;
+    a.tensor_ids = m->d_tensor_ids;
+    a.n_tensors = (uint32_t)m->entries.size();
+    a.seg_count = m->d_seg_count;
+    a.seg_offset = m->d_seg_offset;
+    a.n_segments = m->n_segments;
+    a.out = d_out;
+    a.cap = cap;
+    a.count = d_count;
+    GMS_CUDA(gms::launch_verify(a, static_cast<cudaStream_t>(stream)));
+    return GMS_OK;
+}
+
+int gms_last_device_status(const gms_manifest *m, void *stream, uint64_t *word)
+{
+    if (!m || !word) return GMS_ERR_NULL;
+    if (m->host_only) return GMS_ERR_STATE;
+    unsigned long long w = 0;
+    GMS_CUDA(cudaMemcpyAsync(&w, m->d_status, sizeof w, cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream)));
+    GMS_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    *word = w;
+    return (w & GMS_DEV_TIMEOUT) ? GMS_ERR_TIMEOUT : GMS_OK;
+}
+
+int gms_kv_restore(const gms_kv_pool *pool, const void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
+                   uint32_t image_kind, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
+                   uint64_t *d_kv_digests, uint64_t *d_status, void *stream)
+{
+    if (!pool || !d_status) return GMS_ERR_NULL;
+    if (image_kind != GMS_SRC_DEVICE && image_kind != GMS_SRC_HOST_MAPPED) return GMS_ERR_KIND;
+    if (pool->block_bytes == 0 || pool->block_bytes % gms::kBlockBytes) return GMS_ERR_ALIGN;
+    if (pool->block_bytes > gms::kMaxChunkBlocks * gms::kBlockBytes) return GMS_ERR_ARG;
+    const bool work = n_sel && pool->n_planes;
+    if (work && (!pool->base || !image || !d_block_ids)) return GMS_ERR_NULL;
+    if ((reinterpret_cast<uint64_t>(pool->base) | reinterpret_cast<uint64_t>(image) | pool->plane_stride | pool->block_stride |
+         img_plane_stride | img_slot_stride) & 15u)
+        return GMS_ERR_ALIGN;
+    if (pool->block_stride < pool->block_bytes && pool->n_blocks > 1) return GMS_ERR_ARG;
+    const uint64_t k = pool->block_bytes / gms::kBlockBytes;
+    if ((uint64_t)n_sel * pool->n_planes * k >= 0xffffffffull) return GMS_ERR_RANGE;
+    if (work) {
+        const int rc = check_kind(image, image_kind);
+        if (rc) return rc;
+    }
+    gms::KvArgs a;
+    a.pool_base = static_cast<uint8_t *>(pool->base);
+    a.plane_stride = pool->plane_stride;
+    a.block_stride = pool->block_stride;
+    a.n_planes = pool->n_planes;
+    a.n_blocks = pool->n_blocks;
+    a.block_bytes = pool->block_bytes;
+    a.image = static_cast<const uint8_t *>(image);
+    a.img_plane_stride = img_plane_stride;
+    a.img_slot_stride = img_slot_stride;
+    a.ids = d_block_ids;
+    a.n_sel = n_sel;
+    a.block_digests = d_block_digests;
+    a.kv_digests = d_kv_digests;
+    a.status = reinterpret_cast<unsigned long long *>(d_status);
+    GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
+    return GMS_OK;
+}
+
+int gms_host_image_alloc(uint64_t nbytes, void **host_ptr, void **device_view)
+{
+    if (!host_ptr || !device_view) return GMS_ERR_NULL;
+    *host_ptr = *device_view = nullptr;
+    if (nbytes == 0) return GMS_ERR_ARG;
+    void *h = nullptr, *d = nullptr;
+    cudaError_t e = cudaHostAlloc(&h, nbytes, cudaHostAllocMapped | cudaHostAllocPortable);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : cuda_fail(e);
+    }
+    e = cudaHostGetDevicePointer(&d, h, 0);
+    if (e != cudaSuccess) {
+        cudaFreeHost(h);
+        return cuda_fail(e);
+    }
+    *host_ptr = h;
+    *device_view = d;
+    return GMS_OK;
+}
+
+int gms_host_image_free(void *host_ptr)
+{
+    if (!host_ptr) return GMS_OK;
+    GMS_CUDA(cudaFreeHost(host_ptr));
+    return GMS_OK;
+}
+
+int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *smem_bytes)
+{
+    gms::Geometry g;
+    GMS_CUDA(gms::get_geometry(&g));
+    if (grid_ctas) *grid_ctas = g.grid;
+    if (warps_per_cta) *warps_per_cta = g.warps;
+    if (smem_bytes) *smem_bytes = g.smem;
+    return GMS_OK;
+}
+
+const char *gms_strerror(int status)
+{
+    switch (status) {
+    case GMS_OK: return "ok";
+    case GMS_ERR_NULL: return "a required pointer is NULL";
+    case GMS_ERR_ALIGN: return "offset, pointer or stride is not 16-byte aligned (or block_bytes is not a multiple of 4096)";
+    case GMS_ERR_RANGE: return "range exceeds the image or an index limit";
+    case GMS_ERR_OVERLAP: return "destination ranges overlap";
+    case GMS_ERR_DUP_ID: return "duplicate tensor_id";
+    case GMS_ERR_NOMEM: return "out of memory for the manifest's tables";
+    case GMS_ERR_CUDA: return "a CUDA call failed (see gms_last_cuda_error)";
+    case GMS_ERR_KIND: return "image pointer does not match image_kind";
+    case GMS_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case GMS_ERR_STATE: return "manifest lacks device tables or recorded digests";
+    case GMS_ERR_ARG: return "argument out of range";
+    default: return "unknown status";
+    }
+}
+
+const char *gms_last_cuda_error(void) { return t_cuda_error.c_str(); }
+
+uint32_t gms_version(void) { return 0x00010000u; }
+
+}  // extern "C"

@@ -1,0 +1,80 @@
+// Internal declarations shared by the host API and the kernel translation units.
+// Nothing here is part of the public ABI (that is include/gms.h).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace gms {
+
+constexpr uint32_t kBlockBytes = 4096;     // digest block
+constexpr uint32_t kMaxChunkBlocks = 32;   // one lane keeps one block digest of the chunk in flight
+constexpr uint64_t kG = 0x9E3779B97F4A7C15ull;
+
+// One unit of the persistent kernels' work list: a run of whole digest blocks of
+// one tensor (the last block of a tensor may be short).  32 bytes, read as 2 x 16 B.
+struct alignas(16) Chunk {
+    uint64_t src_off;  // byte offset of the run in the packed image
+    uint64_t dst;      // device address of the run in its destination
+    uint32_t nbytes;   // 1 .. kMaxChunkBlocks * 4096
+    uint32_t tensor;   // entry index (slot of the tensor digest)
+    uint32_t gblock0;  // slot of the run's first block digest
+    uint32_t tblock0;  // index of that block inside the tensor
+};
+static_assert(sizeof(Chunk) == 32, "Chunk must stay 32 bytes");
+
+// Launch shape of the streaming kernels (chosen once per process, per device).
+struct Geometry {
+    uint32_t grid;     // CTAs (a multiple of the SM count)
+    uint32_t warps;    // warps per CTA; every warp runs its own copy pipeline
+    uint32_t stages;   // 4 KiB ring slots per warp
+    uint32_t smem;     // dynamic shared memory per CTA
+};
+cudaError_t get_geometry(Geometry *g);
+
+struct StreamArgs {
+    const Chunk *chunks;
+    uint32_t n_chunks;
+    const uint8_t *image;          // restore: base of the packed image; digest: unused
+    uint64_t *block_digests;       // may be null
+    uint64_t *tensor_digests;      // may be null
+    uint32_t n_tensors;
+    unsigned int *work_counter;    // manifest-owned
+    unsigned long long *status;    // manifest-owned device status word
+};
+
+struct KvArgs {
+    uint8_t *pool_base;
+    uint64_t plane_stride, block_stride;
+    uint32_t n_planes, n_blocks, block_bytes;
+    const uint8_t *image;
+    uint64_t img_plane_stride, img_slot_stride;
+    const int32_t *ids;
+    uint32_t n_sel;
+    uint64_t *block_digests;       // may be null
+    uint64_t *kv_digests;          // may be null
+    unsigned long long *status;    // [0] skipped ids, [1] device status word
+};
+
+cudaError_t launch_restore(const StreamArgs &a, cudaStream_t s);
+cudaError_t launch_digest(const StreamArgs &a, cudaStream_t s);
+cudaError_t launch_kv_restore(const KvArgs &a, cudaStream_t s);
+
+struct VerifyArgs {
+    const uint64_t *computed, *expected;
+    uint64_t n_blocks;
+    const uint64_t *block_base;    // n_tensors + 1 prefix sums (device)
+    const uint64_t *tensor_ids;    // n_tensors (device)
+    uint32_t n_tensors;
+    uint32_t *seg_count;           // n_segments scratch (device)
+    uint64_t *seg_offset;          // n_segments scratch (device)
+    uint32_t n_segments;
+    void *out;                     // gms_mismatch[cap]
+    uint32_t cap;
+    uint64_t *count;
+};
+constexpr uint32_t kVerifySegBlocks = 2048;  // digest slots compared by one CTA
+cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s);
+cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s);
+
+}  // namespace gms

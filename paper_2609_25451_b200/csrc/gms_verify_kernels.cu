@@ -1,0 +1,147 @@
+// gms_verify: compare computed block digests with the recorded ones and emit
+// the differing (tensor_id, block) pairs in ascending (entry position, block)
+// order.  The order is made deterministic by an ordered compaction instead of
+// an atomic append: (1) every CTA counts the differences in its own contiguous
+// segment of digest slots, (2) one CTA turns the per-segment counts into
+// offsets and the grand total, (3) every CTA whose segment has differences
+// (normally none) ranks them with a block-wide scan and writes them at
+// offset + rank.  Traffic is 16 bytes per 4 KiB of payload -- noise next to the
+// streaming kernels -- and no CTA ever waits for another.
+#include "gms_internal.h"
+
+namespace gms {
+namespace {
+
+constexpr uint32_t kThreads = 256;
+constexpr uint32_t kPerThread = kVerifySegBlocks / kThreads;  // 8 consecutive slots per thread
+static_assert(kVerifySegBlocks % kThreads == 0, "segment must divide evenly");
+
+struct Mismatch {
+    uint64_t tensor_id, block;
+};
+
+__device__ __forceinline__ uint32_t diff_mask(const uint64_t *c, const uint64_t *x, uint64_t first, uint64_t n)
+{
+    uint32_t mask = 0;
+#pragma unroll
+    for (uint32_t k = 0; k < kPerThread; ++k) {
+        const uint64_t g = first + k;
+        if (g < n && c[g] != x[g]) mask |= 1u << k;
+    }
+    return mask;
+}
+
+__global__ void __launch_bounds__(kThreads) gms_verify_count_kernel(VerifyArgs a)
+{
+    __shared__ uint32_t warp_sum[kThreads / 32];
+    const uint64_t first = (uint64_t)blockIdx.x * kVerifySegBlocks + (uint64_t)threadIdx.x * kPerThread;
+    uint32_t c = __popc(diff_mask(a.computed, a.expected, first, a.n_blocks));
+    c = __reduce_add_sync(0xffffffffu, c);
+    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = 0;
+        for (uint32_t w = 0; w < kThreads / 32; ++w) t += warp_sum[w];
+        a.seg_count[blockIdx.x] = t;
+    }
+}
+
+// One CTA: exclusive prefix sum of the segment counts, and the total.
+__global__ void __launch_bounds__(1024) gms_verify_scan_kernel(VerifyArgs a)
+{
+    __shared__ uint64_t warp_tot[32];
+    __shared__ uint64_t carry;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t base = 0; base < a.n_segments; base += blockDim.x) {
+        const uint32_t i = base + threadIdx.x;
+        const uint64_t v = i < a.n_segments ? a.seg_count[i] : 0;
+        uint64_t incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint64_t o = __shfl_up_sync(0xffffffffu, incl, d);
+            if ((int)lane >= d) incl += o;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        uint64_t before = carry;
+        for (uint32_t w = 0; w < warp; ++w) before += warp_tot[w];
+        if (i < a.n_segments) a.seg_offset[i] = before + incl - v;
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) carry = before + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *a.count = carry;
+}
+
+__global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
+{
+    if (a.seg_count[blockIdx.x] == 0) return;  // the common case: nothing differs here
+    __shared__ uint32_t warp_sum[kThreads / 32];
+    const uint64_t first = (uint64_t)blockIdx.x * kVerifySegBlocks + (uint64_t)threadIdx.x * kPerThread;
+    const uint32_t mask = diff_mask(a.computed, a.expected, first, a.n_blocks);
+    const uint32_t mine = __popc(mask), lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
+        if ((int)lane >= d) incl += o;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    uint64_t rank = a.seg_offset[blockIdx.x] + incl - mine;
+    for (uint32_t w = 0; w < warp; ++w) rank += warp_sum[w];
+    if (!mask) return;
+    Mismatch *out = static_cast<Mismatch *>(a.out);
+    for (uint32_t k = 0; k < kPerThread; ++k) {
+        if (!(mask & (1u << k))) continue;
+        if (rank < a.cap) {
+            const uint64_t g = first + k;
+            // entry t with block_base[t] <= g < block_base[t+1]; empty tensors share a base and are skipped
+            uint32_t lo = 0, hi = a.n_tensors;
+            while (hi - lo > 1) {
+                const uint32_t mid = lo + (hi - lo) / 2;
+                if (a.block_base[mid] <= g) lo = mid; else hi = mid;
+            }
+            out[rank].tensor_id = a.tensor_ids[lo];
+            out[rank].block = g - a.block_base[lo];
+        }
+        ++rank;
+    }
+}
+
+__global__ void gms_copy_u64_kernel(uint64_t *dst, const uint64_t *src, uint64_t n)
+{
+    const uint64_t step = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += step) dst[i] = src[i];
+}
+
+}  // namespace
+
+cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
+{
+    if (a.n_segments == 0) {  // no digest slots at all: count = 0
+        VerifyArgs z = a;
+        gms_verify_scan_kernel<<<1, 32, 0, s>>>(z);
+        return cudaGetLastError();
+    }
+    gms_verify_count_kernel<<<a.n_segments, kThreads, 0, s>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e) return e;
+    gms_verify_scan_kernel<<<1, 1024, 0, s>>>(a);
+    if ((e = cudaGetLastError())) return e;
+    gms_verify_emit_kernel<<<a.n_segments, kThreads, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s)
+{
+    if (n == 0) return cudaSuccess;
+    uint64_t blocks = (n + 1023) / 1024;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    gms_copy_u64_kernel<<<(uint32_t)blocks, 256, 0, s>>>(dst, src, n);
+    return cudaGetLastError();
+}
+
+}  // namespace gms

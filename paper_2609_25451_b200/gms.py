@@ -1,0 +1,220 @@
+"""Thin ctypes binding of the C ABI in ``include/gms.h`` -- argument marshalling only.
+
+Every function has the name and meaning of the C entry point.  Device buffers
+may be passed as ``torch`` tensors (their ``data_ptr()`` is taken), as ints, or
+as ``None`` where the C ABI accepts NULL.  Nothing here computes anything: if
+the shared library is missing or a call fails, an exception is raised -- there
+is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libgms.so")
+
+BLOCK_BYTES = 4096
+OK = 0
+ERR_NULL, ERR_ALIGN, ERR_RANGE, ERR_OVERLAP, ERR_DUP_ID, ERR_NOMEM = -1, -2, -3, -4, -5, -6
+ERR_CUDA, ERR_KIND, ERR_TIMEOUT, ERR_STATE, ERR_ARG = -7, -8, -9, -10, -11
+SRC_DEVICE, SRC_HOST_MAPPED = 0, 1
+BUILD_HOST_ONLY = 1
+
+# numpy view of gms_entry / gms_mismatch (32 and 16 bytes)
+ENTRY_DTYPE = np.dtype([("tensor_id", "<u8"), ("src_offset", "<u8"), ("dst", "<u8"), ("nbytes", "<u8")])
+MISMATCH_DTYPE = np.dtype([("tensor_id", "<u8"), ("block", "<u8")])
+
+EXPORTS = (
+    "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
+    "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_digest",
+    "gms_verify", "gms_last_device_status", "gms_kv_restore", "gms_host_image_alloc", "gms_host_image_free",
+    "gms_launch_geometry", "gms_strerror", "gms_last_cuda_error", "gms_version",
+)
+
+
+class GmsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        text = lib().gms_strerror(status).decode()
+        if status == ERR_CUDA:
+            text += " -- " + lib().gms_last_cuda_error().decode()
+        super().__init__(f"{where}: {text} ({status})")
+
+
+class KvPool(C.Structure):
+    _fields_ = [("base", C.c_void_p), ("plane_stride", C.c_uint64), ("block_stride", C.c_uint64),
+                ("n_planes", C.c_uint32), ("n_blocks", C.c_uint32), ("block_bytes", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads ``libgms.so`` (built by ``paper_2609_25451_b200.build``); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2609_25451_b200.build` (needs nvcc)")
+        L = C.CDLL(LIB_PATH)
+        p, u64, u32, i = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int
+        pp = C.POINTER(C.c_void_p)
+        pu64, pu32 = C.POINTER(C.c_uint64), C.POINTER(C.c_uint32)
+        sig = {
+            "gms_manifest_build": (i, [p, C.c_size_t, u64, u32, pp]),
+            "gms_manifest_destroy": (i, [p]),
+            "gms_manifest_info": (i, [p, pu64, pu64, pu64]),
+            "gms_manifest_block_base": (i, [p, C.c_size_t, pu64]),
+            "gms_manifest_chunk_count": (i, [p, pu64]),
+            "gms_manifest_chunk": (i, [p, u64, pu64, pu64, pu64]),
+            "gms_manifest_set_expected": (i, [p, p, p]),
+            "gms_restore": (i, [p, p, u32, p, p, p]),
+            "gms_digest": (i, [p, p, p, p]),
+            "gms_verify": (i, [p, p, p, u32, p, p]),
+            "gms_last_device_status": (i, [p, p, pu64]),
+            "gms_kv_restore": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
+            "gms_host_image_alloc": (i, [u64, pp, pp]),
+            "gms_host_image_free": (i, [p]),
+            "gms_launch_geometry": (i, [pu32, pu32, pu32]),
+            "gms_strerror": (C.c_char_p, [i]),
+            "gms_last_cuda_error": (C.c_char_p, []),
+            "gms_version": (u32, []),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _dev(x):
+    """Address of a device buffer: torch tensor, int or None."""
+    if x is None:
+        return None
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    return int(x)
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
+    return getattr(stream, "cuda_stream", stream)
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise GmsError(rc, where)
+
+
+def make_entries(rows) -> np.ndarray:
+    """rows: iterable of (tensor_id, src_offset, dst_address, nbytes) -> gms_entry array."""
+    rows = list(rows)
+    a = np.zeros(len(rows), dtype=ENTRY_DTYPE)
+    for k, r in enumerate(rows):
+        a[k] = tuple(int(v) for v in r)
+    return a
+
+
+class Manifest:
+    """Owner of a ``gms_manifest*``; destroyed on ``close()`` / garbage collection."""
+
+    def __init__(self, handle):
+        self.handle = handle
+        n, nb, pay = C.c_uint64(), C.c_uint64(), C.c_uint64()
+        _check(lib().gms_manifest_info(handle, C.byref(n), C.byref(nb), C.byref(pay)), "gms_manifest_info")
+        self.n_tensors, self.n_blocks, self.payload_bytes = n.value, nb.value, pay.value
+
+    def close(self):
+        if self.handle:
+            lib().gms_manifest_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+
+def gms_manifest_build(entries, image_bytes: int, flags: int = 0) -> Manifest:
+    e = np.ascontiguousarray(entries, dtype=ENTRY_DTYPE)
+    out = C.c_void_p()
+    rc = lib().gms_manifest_build(e.ctypes.data if len(e) else None, len(e), int(image_bytes), int(flags), C.byref(out))
+    _check(rc, "gms_manifest_build")
+    return Manifest(out.value)
+
+
+def gms_manifest_block_base(m: Manifest, entry_index: int) -> int:
+    v = C.c_uint64()
+    _check(lib().gms_manifest_block_base(m.handle, entry_index, C.byref(v)), "gms_manifest_block_base")
+    return v.value
+
+
+def gms_manifest_chunk_count(m: Manifest) -> int:
+    v = C.c_uint64()
+    _check(lib().gms_manifest_chunk_count(m.handle, C.byref(v)), "gms_manifest_chunk_count")
+    return v.value
+
+
+def gms_manifest_chunk(m: Manifest, i: int):
+    """Returns (entry_index, tensor_byte_offset, nbytes) of work-list chunk ``i``."""
+    a, b, c = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    _check(lib().gms_manifest_chunk(m.handle, i, C.byref(a), C.byref(b), C.byref(c)), "gms_manifest_chunk")
+    return a.value, b.value, c.value
+
+
+def gms_manifest_set_expected(m: Manifest, d_block_digests, stream=None):
+    _check(lib().gms_manifest_set_expected(m.handle, _dev(d_block_digests), _stream(stream)), "gms_manifest_set_expected")
+
+
+def gms_restore(m: Manifest, image, image_kind: int, d_block_digests, d_tensor_digests, stream=None):
+    _check(lib().gms_restore(m.handle, _dev(image), image_kind, _dev(d_block_digests), _dev(d_tensor_digests),
+                             _stream(stream)), "gms_restore")
+
+
+def gms_digest(m: Manifest, d_block_digests, d_tensor_digests, stream=None):
+    _check(lib().gms_digest(m.handle, _dev(d_block_digests), _dev(d_tensor_digests), _stream(stream)), "gms_digest")
+
+
+def gms_verify(m: Manifest, d_block_digests, d_out, cap: int, d_count, stream=None):
+    _check(lib().gms_verify(m.handle, _dev(d_block_digests), _dev(d_out), cap, _dev(d_count), _stream(stream)), "gms_verify")
+
+
+def gms_last_device_status(m: Manifest, stream=None) -> int:
+    w = C.c_uint64()
+    _check(lib().gms_last_device_status(m.handle, _stream(stream), C.byref(w)), "gms_last_device_status")
+    return w.value
+
+
+def gms_kv_restore(pool: KvPool, image, img_plane_stride: int, img_slot_stride: int, image_kind: int, d_block_ids,
+                   n_sel: int, d_block_digests, d_kv_digests, d_status, stream=None):
+    _check(lib().gms_kv_restore(C.byref(pool), _dev(image), img_plane_stride, img_slot_stride, image_kind,
+                                _dev(d_block_ids), n_sel, _dev(d_block_digests), _dev(d_kv_digests), _dev(d_status),
+                                _stream(stream)), "gms_kv_restore")
+
+
+def gms_host_image_alloc(nbytes: int):
+    """Returns (host_ptr, device_view, numpy uint8 array over the pinned mapping)."""
+    h, d = C.c_void_p(), C.c_void_p()
+    _check(lib().gms_host_image_alloc(int(nbytes), C.byref(h), C.byref(d)), "gms_host_image_alloc")
+    arr = np.ctypeslib.as_array((C.c_uint8 * int(nbytes)).from_address(h.value))
+    return h.value, d.value, arr
+
+
+def gms_host_image_free(host_ptr: int):
+    _check(lib().gms_host_image_free(host_ptr), "gms_host_image_free")
+
+
+def gms_launch_geometry():
+    g, w, s = C.c_uint32(), C.c_uint32(), C.c_uint32()
+    _check(lib().gms_launch_geometry(C.byref(g), C.byref(w), C.byref(s)), "gms_launch_geometry")
+    return {"grid_ctas": g.value, "warps_per_cta": w.value, "smem_bytes": s.value}
+
+
+def gms_strerror(status: int) -> str:
+    return lib().gms_strerror(status).decode()
+
+
+def gms_version() -> int:
+    return lib().gms_version()

@@ -1,0 +1,254 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU oracle on the same
+seeded inputs -- element by element, bit-exact (everything here is integer work): destination
+bytes, block digests, tensor digests, mismatch lists and counts, KV status counts.  Sizes are
+small enough for the oracle yet span many chunks, several ring slots per warp and ragged tails.
+Guard bands around every destination and canary words around every output array catch stray writes."""
+import ctypes
+import zlib
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+from paper_2609_25451_b200 import gms  # noqa: E402
+from paper_2609_25451_b200 import workloads as W  # noqa: E402
+
+from gpu_harness import CANARY, FILL, PAD, DeviceWorkload, guarded_u64, oracle_record, payload_of  # noqa: E402
+
+EDGE_SIZES = [0, 1, 7, 8, 9, 15, 16, 17, 31, 4080, 4095, 4096, 4097, 4111, 4112, 8191, 8192, 8193, 0, 12288,
+              65535, 65536, 65537, 131071, 131072, 131073, 262144 + 5, 1 << 20, (1 << 20) + 4097, 3, 0]
+
+WORKLOADS = {
+    "tiny64": lambda: W.tiny_manifest(),
+    "edge": lambda: W.pack_layout("edge", EDGE_SIZES, seed=11),
+    "mixed-odd": lambda: W.mixed_manifest(n_small=3000, n_large=2, large_bytes=(8 << 20) + 24, round16=False),
+    "llama8b/16": lambda: W.llama3_8b_manifest(shrink=16),
+}
+
+
+def oracle_restore(oracle, w, image):
+    slab = np.full(w.slab_bytes, FILL, np.uint8)
+    rc, bd, td = oracle.restore(oracle_record(oracle, w), image, slab)
+    assert rc == 0
+    return slab, bd, td
+
+
+@pytest.mark.parametrize("name", sorted(WORKLOADS))
+def test_restore_digest_verify_parity(oracle, name):
+    w = WORKLOADS[name]()
+    image = W.random_bytes_host(w.image_bytes, seed=zlib.crc32(name.encode()) & 0xFFFF)
+    want_slab, want_bd, want_td = oracle_restore(oracle, w, image)
+    d = DeviceWorkload(w, image)
+
+    bd, td = d.restore()
+    got_slab = d.slab_host()
+    assert np.array_equal(got_slab, want_slab), "destination bytes (or guard bands) differ"
+    assert np.array_equal(bd, want_bd) and np.array_equal(td, want_td)
+
+    # digest in place: same digests, destinations untouched
+    bd2, td2 = d.digest()
+    assert np.array_equal(bd2, want_bd) and np.array_equal(td2, want_td)
+    assert np.array_equal(d.slab_host(), want_slab)
+
+    # record the digests; a clean verify reports nothing
+    gms.gms_manifest_set_expected(d.m, d.bd_ptr())
+    assert d.verify(cap=8) == (0, [])
+
+    # host-made single-bit flips are named exactly, in (entry, block) order
+    flips = W.flip_positions(w, 3, seed=5)
+    rec = oracle_record(oracle, w)
+    for row, byte, bit in flips:
+        d.flip(row, byte, bit)
+        want_slab[int(w.rows[row]["dst_offset"]) + byte] ^= 1 << bit
+    bd3, td3 = d.digest()
+    _, obd3, otd3 = oracle.digest(rec, want_slab)
+    assert np.array_equal(bd3, obd3) and np.array_equal(td3, otd3)
+    count, pairs = d.verify(cap=8)
+    ocount, omm = oracle.verify(rec, obd3, want_bd, cap=8)
+    assert count == ocount == 3
+    assert pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+    assert sorted(pairs) == sorted((int(w.rows[r]["tensor_id"]), b // 4096) for r, b, _ in flips)
+    # cap smaller than the count: total still reported, only cap entries written
+    count, pairs = d.verify(cap=2)
+    assert count == 3 and pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm][:2]
+    count, pairs = d.verify(cap=0)
+    assert count == 3 and pairs == []
+    d.close()
+
+
+def test_optional_outputs_may_be_null(oracle):
+    w = W.pack_layout("opt", [5000, 70000, 16, 0, 4096], seed=3)
+    image = W.random_bytes_host(w.image_bytes, seed=8)
+    want_slab, want_bd, want_td = oracle_restore(oracle, w, image)
+    d = DeviceWorkload(w, image)
+    for want_b, want_t in ((True, False), (False, True), (False, False)):
+        d.slab.fill_(FILL)
+        bd, td = d.restore(want_bd=want_b, want_td=want_t)
+        assert np.array_equal(d.slab_host(), want_slab)
+        assert np.array_equal(bd, want_bd) if want_b else (bd == CANARY).all()
+        assert np.array_equal(td, want_td) if want_t else (td == CANARY).all()
+    d.close()
+
+
+def test_empty_manifests(oracle):
+    for sizes in ([], [0, 0, 0]):
+        w = W.pack_layout("empty", sizes, seed=1)
+        d = DeviceWorkload(w, np.zeros(w.image_bytes, np.uint8))
+        bd, td = d.restore()
+        assert bd.size == 0 and (td == 0).all() and td.size == len(sizes)
+        bd, td = d.digest()
+        assert (td == 0).all()
+        gms.gms_manifest_set_expected(d.m, d.bd_ptr())
+        assert d.verify(cap=4) == (0, [])
+        assert (d.slab_host() == FILL).all()
+        d.close()
+
+
+def test_results_do_not_depend_on_entry_order_or_chunking(oracle, monkeypatch):
+    w = W.mixed_manifest(n_small=800, n_large=1, large_bytes=5 << 20, round16=False, seed=77)
+    image = W.random_bytes_host(w.image_bytes, seed=9)
+    d = DeviceWorkload(w, image)
+    bd, td = d.restore()
+    slab = d.slab_host()
+    by_id = {int(r["tensor_id"]): int(td[t]) for t, r in enumerate(w.rows)}
+    d.close()
+    # permuted entries: per-id results unchanged, destination bytes identical
+    perm = np.random.default_rng(5).permutation(len(w.rows))
+    w2 = W.Workload(w.name, w.rows[perm].copy(), w.image_bytes, w.slab_bytes)
+    d2 = DeviceWorkload(w2, image)
+    bd2, td2 = d2.restore()
+    assert np.array_equal(d2.slab_host(), slab)
+    assert {int(r["tensor_id"]): int(td2[t]) for t, r in enumerate(w2.rows)} == by_id
+    d2.close()
+    # different internal chunk length: every output bit-identical
+    for blocks in ("1", "5", "32"):
+        monkeypatch.setenv("GMS_CHUNK_BLOCKS", blocks)
+        d3 = DeviceWorkload(w, image)
+        bd3, td3 = d3.restore()
+        assert np.array_equal(bd3, bd) and np.array_equal(td3, td) and np.array_equal(d3.slab_host(), slab)
+        d3.close()
+
+
+def test_many_mismatches_exceed_cap_in_order(oracle):
+    w = W.pack_layout("many", [4096 * 700 + 100, 4096 * 3000, 10, 4096 * 5000 + 1], seed=2)
+    image = W.random_bytes_host(w.image_bytes, seed=10)
+    rec = oracle_record(oracle, w)
+    d = DeviceWorkload(w, image)
+    want_slab, want_bd, _ = oracle_restore(oracle, w, image)
+    d.restore()
+    gms.gms_manifest_set_expected(d.m, d.bd_ptr())
+    # corrupt every 3rd block of the slab region wholesale (host-made corruption)
+    rng = np.random.default_rng(4)
+    for row in range(len(w.rows)):
+        nb = int(w.rows[row]["nbytes"])
+        for b in range(0, (nb + 4095) // 4096, 3):
+            pos = int(w.rows[row]["dst_offset"]) + min(nb - 1, b * 4096 + int(rng.integers(0, 4096)))
+            want_slab[pos] ^= 0x10
+    d.slab.copy_(torch.from_numpy(want_slab))
+    bd, _ = d.digest()
+    _, obd, _ = oracle.digest(rec, want_slab)
+    assert np.array_equal(bd, obd)
+    for cap in (100, 5000):
+        count, pairs = d.verify(cap=cap)
+        ocount, omm = oracle.verify(rec, obd, want_bd, cap=cap)
+        assert count == ocount and count > 2500
+        assert pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+    d.close()
+
+
+def test_host_mapped_source_parity(oracle):
+    w = W.mixed_manifest(n_small=400, n_large=1, large_bytes=(2 << 20) + 40, round16=False, seed=31)
+    image = W.random_bytes_host(w.image_bytes, seed=12)
+    want_slab, want_bd, want_td = oracle_restore(oracle, w, image)
+    hptr, dview, arr = gms.gms_host_image_alloc(w.image_bytes)
+    try:
+        arr[:] = image
+        d = DeviceWorkload(w, image)
+        bd, td = d.restore(image=dview, kind=gms.SRC_HOST_MAPPED)
+        assert np.array_equal(d.slab_host(), want_slab)
+        assert np.array_equal(bd, want_bd) and np.array_equal(td, want_td)
+        # the pointer must be what image_kind says
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_restore(d.m, dview, gms.SRC_DEVICE, None, None)
+        assert ei.value.status == gms.ERR_KIND
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_restore(d.m, d.image, gms.SRC_HOST_MAPPED, None, None)
+        assert ei.value.status == gms.ERR_KIND
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_restore(d.m, d.image.data_ptr() + 8, gms.SRC_DEVICE, None, None)
+        assert ei.value.status == gms.ERR_ALIGN
+        d.close()
+    finally:
+        torch.cuda.synchronize()
+        gms.gms_host_image_free(hptr)
+
+
+def run_kv(oracle, n_planes, n_blocks, block_bytes, ids, plane_gap, seed, host_mapped=False):
+    k = block_bytes // 4096
+    plane_stride = n_blocks * block_bytes + plane_gap
+    n_sel = len(ids)
+    ips, iss = max(n_sel, 1) * block_bytes + 64, block_bytes
+    pool_h = W.random_bytes_host(n_planes * plane_stride, seed)
+    img_h = W.random_bytes_host(n_planes * ips, seed + 1)
+    want_pool = pool_h.copy()
+    rc, obd, okd, oskip = oracle.kv_restore(want_pool, plane_stride, block_bytes, n_planes, n_blocks, block_bytes, img_h,
+                                            ips, iss, ids)
+    assert rc == 0
+    pool = torch.from_numpy(pool_h).cuda()
+    hptr = None
+    if host_mapped:
+        hptr, img_ptr, arr = gms.gms_host_image_alloc(img_h.size)
+        arr[:] = img_h
+    else:
+        img = torch.from_numpy(img_h).cuda()
+        img_ptr = img.data_ptr()
+    ids_d = torch.from_numpy(np.ascontiguousarray(ids, dtype=np.int32)).cuda()
+    bd, kd, st = guarded_u64(n_sel * n_planes * k), guarded_u64(n_sel), guarded_u64(2)
+    desc = gms.KvPool(base=pool.data_ptr(), plane_stride=plane_stride, block_stride=block_bytes, n_planes=n_planes,
+                      n_blocks=n_blocks, block_bytes=block_bytes)
+    gms.gms_kv_restore(desc, img_ptr, ips, iss, gms.SRC_HOST_MAPPED if host_mapped else gms.SRC_DEVICE, ids_d, n_sel,
+                       bd.data_ptr() + 8 * PAD, kd.data_ptr() + 8 * PAD, st.data_ptr() + 8 * PAD)
+    torch.cuda.synchronize()
+    status = payload_of(st, 2)
+    assert int(status[0]) == oskip and int(status[1]) == 0
+    assert np.array_equal(pool.cpu().numpy(), want_pool), "pool bytes differ"
+    assert np.array_equal(payload_of(bd, n_sel * n_planes * k), obd)
+    assert np.array_equal(payload_of(kd, n_sel), okd)
+    if hptr:
+        gms.gms_host_image_free(hptr)
+
+
+def test_kv_restore_parity(oracle):
+    rng = np.random.default_rng(41)
+    ids = rng.permutation(300)[:90].astype(np.int32)
+    run_kv(oracle, n_planes=6, n_blocks=300, block_bytes=32768, ids=ids, plane_gap=4096, seed=50)
+
+
+def test_kv_restore_out_of_range_ids_are_skipped_and_counted(oracle):
+    ids = np.array([5, -1, 0, 40, 39, 2**31 - 1, -(2**31), 7], np.int32)
+    run_kv(oracle, n_planes=4, n_blocks=40, block_bytes=8192, ids=ids, plane_gap=0, seed=60)
+
+
+def test_kv_restore_other_block_sizes_and_host_source(oracle):
+    rng = np.random.default_rng(43)
+    run_kv(oracle, 3, 64, 4096, rng.permutation(64)[:20].astype(np.int32), 256, 70)
+    run_kv(oracle, 2, 16, 131072, rng.permutation(16)[:9].astype(np.int32), 0, 80)
+    run_kv(oracle, 5, 50, 32768, rng.permutation(50)[:11].astype(np.int32), 512, 90, host_mapped=True)
+    run_kv(oracle, 5, 50, 32768, np.zeros(0, np.int32), 0, 95)
+
+
+def test_geometry_is_a_multiple_of_the_sm_count():
+    g = gms.gms_launch_geometry()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert g["grid_ctas"] % sms == 0 and g["warps_per_cta"] >= 1 and g["smem_bytes"] <= 227 * 1024
+
+
+def test_product_path_does_not_import_the_oracle():
+    import paper_2609_25451_b200.gms as g
+
+    src = open(g.__file__).read()
+    assert "import oracle" not in src and "from oracle" not in src and "gms_oracle" not in src
+    assert isinstance(ctypes.CDLL(g.LIB_PATH), ctypes.CDLL)
