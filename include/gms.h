@@ -223,6 +223,14 @@ int gms_host_image_free(void *host_ptr);
 
 /* Launch geometry of the streaming kernels on the current device (for reporting). */
 int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *smem_bytes);
+/* Number of kernels this library has launched in this process so far (for reporting). */
+uint64_t gms_kernel_launches(void);
+/*
+ * Makes `device` current for the calling thread's later gms_* calls.  The library links its own
+ * copy of the CUDA runtime; a process that drives several GPUs (one service per GPU, Section 4)
+ * selects the device here as well as in whatever else it uses.
+ */
+int gms_set_device(int device);
 
 const char *gms_strerror(int status);
 const char *gms_last_cuda_error(void); /* text of the last failed CUDA call on this thread */

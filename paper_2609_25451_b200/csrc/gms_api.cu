@@ -3,6 +3,7 @@
 // points that enqueue the kernels.  There is no CPU implementation of the data
 // path here: every entry point either launches the CUDA kernels or fails.
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -36,6 +37,7 @@ struct gms_manifest {
 
 namespace {
 
+std::atomic<uint64_t> g_launches{0};
 thread_local std::string t_cuda_error;
 
 int cuda_fail(cudaError_t e)
@@ -88,6 +90,10 @@ int check_kind(const void *image, uint32_t kind)
 }
 
 }  // namespace
+
+namespace gms {
+void count_launches(uint32_t n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace gms
 
 extern "C" {
 
@@ -411,6 +417,14 @@ int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *
     if (grid_ctas) *grid_ctas = g.grid;
     if (warps_per_cta) *warps_per_cta = g.warps;
     if (smem_bytes) *smem_bytes = g.smem;
+    return GMS_OK;
+}
+
+uint64_t gms_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int gms_set_device(int device)
+{
+    GMS_CUDA(cudaSetDevice(device));
     return GMS_OK;
 }
 

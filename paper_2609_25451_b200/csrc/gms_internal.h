@@ -77,4 +77,6 @@ constexpr uint32_t kVerifySegBlocks = 2048;  // digest slots compared by one CTA
 cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s);
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s);
 
+void count_launches(uint32_t n);  // bumps the process-wide launch counter
+
 }  // namespace gms

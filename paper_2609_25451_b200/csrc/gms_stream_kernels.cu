@@ -410,6 +410,7 @@ cudaError_t prologue(uint64_t *accum, uint64_t n_accum, unsigned int *counter, u
     if (blocks < 1) blocks = 1;
     if (blocks > 1184) blocks = 1184;
     gms_prologue_kernel<<<(uint32_t)blocks, threads, 0, s>>>(accum, n_accum, counter, status, n_status);
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -427,6 +428,7 @@ cudaError_t launch_stream(const StreamArgs &a, cudaStream_t s)
     case 8: gms_stream_kernel<8, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
     default: gms_stream_kernel<4, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
     }
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -483,6 +485,7 @@ cudaError_t launch_kv_restore(const KvArgs &a, cudaStream_t s)
     case 8: gms_kv_stream_kernel<8><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
     default: gms_kv_stream_kernel<4><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
     }
+    count_launches(1);
     return cudaGetLastError();
 }
 

@@ -124,6 +124,7 @@ cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
     if (a.n_segments == 0) {  // no digest slots at all: count = 0
         VerifyArgs z = a;
         gms_verify_scan_kernel<<<1, 32, 0, s>>>(z);
+        count_launches(1);
         return cudaGetLastError();
     }
     gms_verify_count_kernel<<<a.n_segments, kThreads, 0, s>>>(a);
@@ -132,6 +133,7 @@ cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
     gms_verify_scan_kernel<<<1, 1024, 0, s>>>(a);
     if ((e = cudaGetLastError())) return e;
     gms_verify_emit_kernel<<<a.n_segments, kThreads, 0, s>>>(a);
+    count_launches(3);
     return cudaGetLastError();
 }
 
@@ -141,6 +143,7 @@ cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cuda
     uint64_t blocks = (n + 1023) / 1024;
     if (blocks > 148 * 8) blocks = 148 * 8;
     gms_copy_u64_kernel<<<(uint32_t)blocks, 256, 0, s>>>(dst, src, n);
+    count_launches(1);
     return cudaGetLastError();
 }
 

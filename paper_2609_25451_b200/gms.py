@@ -31,7 +31,7 @@ EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_digest",
     "gms_verify", "gms_last_device_status", "gms_kv_restore", "gms_host_image_alloc", "gms_host_image_free",
-    "gms_launch_geometry", "gms_strerror", "gms_last_cuda_error", "gms_version",
+    "gms_launch_geometry", "gms_kernel_launches", "gms_set_device", "gms_strerror", "gms_last_cuda_error", "gms_version",
 )
 
 
@@ -78,6 +78,8 @@ def lib():
             "gms_host_image_alloc": (i, [u64, pp, pp]),
             "gms_host_image_free": (i, [p]),
             "gms_launch_geometry": (i, [pu32, pu32, pu32]),
+            "gms_kernel_launches": (u64, []),
+            "gms_set_device": (i, [i]),
             "gms_strerror": (C.c_char_p, [i]),
             "gms_last_cuda_error": (C.c_char_p, []),
             "gms_version": (u32, []),
@@ -210,6 +212,14 @@ def gms_launch_geometry():
     g, w, s = C.c_uint32(), C.c_uint32(), C.c_uint32()
     _check(lib().gms_launch_geometry(C.byref(g), C.byref(w), C.byref(s)), "gms_launch_geometry")
     return {"grid_ctas": g.value, "warps_per_cta": w.value, "smem_bytes": s.value}
+
+
+def gms_kernel_launches() -> int:
+    return int(lib().gms_kernel_launches())
+
+
+def gms_set_device(device: int):
+    _check(lib().gms_set_device(int(device)), "gms_set_device")
 
 
 def gms_strerror(status: int) -> str:
