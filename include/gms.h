@@ -75,6 +75,7 @@ extern "C" {
 #define GMS_ERR_TIMEOUT (-9)  /* a bounded device-side wait gave up (see device status word)  */
 #define GMS_ERR_STATE (-10)   /* manifest has no device tables / no recorded digests          */
 #define GMS_ERR_ARG (-11)     /* an argument is out of its documented range                   */
+#define GMS_ERR_TOO_LARGE (-12) /* more digest blocks than gms_verify_flat_noalloc has room for */
 
 /* where the packed snapshot image lives */
 #define GMS_SRC_DEVICE 0u      /* device memory (a staging buffer in HBM)                     */
@@ -174,6 +175,37 @@ int gms_digest(const gms_manifest *m, uint64_t *d_block_digests, uint64_t *d_ten
  */
 int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_mismatch *d_out, uint32_t cap,
                uint64_t *d_count, void *stream);
+
+/*
+ * gms_verify_flat_noalloc -- the paper has no counterpart; this is a convenience of this library.
+ *
+ * Who it is for.  Some callers of a memory service cannot allocate device memory at the moment
+ * they need the trust decision: a checker that attaches to a GPU whose memory has already been
+ * handed out in full (service slabs plus an engine's KV pool leave no room, so cudaMalloc would
+ * fail), or a watchdog that must not enter the allocator because an allocation can stall behind,
+ * or disturb, the engine that is serving on the same device.  gms_verify needs a manifest, and
+ * building one allocates.  This entry point compares two digest arrays the caller already holds
+ * and allocates nothing: no cudaMalloc, no cudaFree, no allocating library call.  Its working
+ * tables (per-segment counts and offsets of the ordered compaction) live in a fixed array of about
+ * 24 KiB inside the library image, present on every GPU that loads the library until the process
+ * exits.
+ *
+ * What it computes.  Exactly what gms_verify reports for a manifest with the single entry
+ * (tensor_id, nbytes = n_blocks * 4096): the pairs (tensor_id, b) with
+ * d_computed[b] != d_expected[b], ascending in b, into d_out (device, `cap` slots), and the total
+ * number of differing blocks into *d_count (device), which may exceed cap.
+ *   d_computed, d_expected  (device) n_blocks u64 each
+ *   n_blocks                at most GMS_NOALLOC_MAX_BLOCKS (16 GiB of payload); more is refused
+ *                           with GMS_ERR_TOO_LARGE before anything is enqueued
+ * Rules.  The first call on a device looks up the device address of the fixed array (a one-time
+ * set-up with that device current); make that first call before starting any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's contents (each call
+ * rewrites what it uses before use): two calls that overlap on the GPU race, so keep them on one
+ * stream or order them with events.  Errors: NULL, TOO_LARGE, ARG, CUDA.
+ */
+#define GMS_NOALLOC_MAX_BLOCKS 4194304ull
+int gms_verify_flat_noalloc(const uint64_t *d_computed, const uint64_t *d_expected, uint64_t n_blocks, uint64_t tensor_id,
+                            gms_mismatch *d_out, uint32_t cap, uint64_t *d_count, void *stream);
 
 /* Device status word of the manifest's last call (synchronises `stream`). 0 = clean. */
 int gms_last_device_status(const gms_manifest *m, void *stream, uint64_t *word);

@@ -93,6 +93,7 @@ int check_kind(const void *image, uint32_t kind)
 
 namespace gms {
 void count_launches(uint32_t n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+int report_cuda_error(cudaError_t e) { return cuda_fail(e); }
 }  // namespace gms
 
 extern "C" {
@@ -443,6 +444,7 @@ const char *gms_strerror(int status)
     case GMS_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case GMS_ERR_STATE: return "manifest lacks device tables or recorded digests";
     case GMS_ERR_ARG: return "argument out of range";
+    case GMS_ERR_TOO_LARGE: return "size exceeds the fixed capacity of the no-allocation entry point (GMS_NOALLOC_MAX_BLOCKS)";
     default: return "unknown status";
     }
 }

@@ -78,5 +78,6 @@ cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s);
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s);
 
 void count_launches(uint32_t n);  // bumps the process-wide launch counter
+int report_cuda_error(cudaError_t e);  // records the text for gms_last_cuda_error(); returns GMS_ERR_CUDA
 
 }  // namespace gms

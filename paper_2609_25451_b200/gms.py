@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_PKG, "libgms.so")
 BLOCK_BYTES = 4096
 OK = 0
 ERR_NULL, ERR_ALIGN, ERR_RANGE, ERR_OVERLAP, ERR_DUP_ID, ERR_NOMEM = -1, -2, -3, -4, -5, -6
-ERR_CUDA, ERR_KIND, ERR_TIMEOUT, ERR_STATE, ERR_ARG = -7, -8, -9, -10, -11
+ERR_CUDA, ERR_KIND, ERR_TIMEOUT, ERR_STATE, ERR_ARG, ERR_TOO_LARGE = -7, -8, -9, -10, -11, -12
+NOALLOC_MAX_BLOCKS = 4194304
 SRC_DEVICE, SRC_HOST_MAPPED = 0, 1
 BUILD_HOST_ONLY = 1
 
@@ -30,7 +31,7 @@ MISMATCH_DTYPE = np.dtype([("tensor_id", "<u8"), ("block", "<u8")])
 EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_digest",
-    "gms_verify", "gms_last_device_status", "gms_kv_restore", "gms_host_image_alloc", "gms_host_image_free",
+    "gms_verify", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_host_image_alloc", "gms_host_image_free",
     "gms_launch_geometry", "gms_kernel_launches", "gms_set_device", "gms_strerror", "gms_last_cuda_error", "gms_version",
 )
 
@@ -73,6 +74,7 @@ def lib():
             "gms_restore": (i, [p, p, u32, p, p, p]),
             "gms_digest": (i, [p, p, p, p]),
             "gms_verify": (i, [p, p, p, u32, p, p]),
+            "gms_verify_flat_noalloc": (i, [p, p, u64, u64, p, u32, p, p]),
             "gms_last_device_status": (i, [p, p, pu64]),
             "gms_kv_restore": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
             "gms_host_image_alloc": (i, [u64, pp, pp]),
@@ -181,6 +183,12 @@ def gms_digest(m: Manifest, d_block_digests, d_tensor_digests, stream=None):
 
 def gms_verify(m: Manifest, d_block_digests, d_out, cap: int, d_count, stream=None):
     _check(lib().gms_verify(m.handle, _dev(d_block_digests), _dev(d_out), cap, _dev(d_count), _stream(stream)), "gms_verify")
+
+
+def gms_verify_flat_noalloc(d_computed, d_expected, n_blocks: int, tensor_id: int, d_out, cap: int, d_count, stream=None):
+    """Allocation-free comparison of two device digest arrays; see include/gms.h for who needs it."""
+    _check(lib().gms_verify_flat_noalloc(_dev(d_computed), _dev(d_expected), int(n_blocks), int(tensor_id), _dev(d_out),
+                                         cap, _dev(d_count), _stream(stream)), "gms_verify_flat_noalloc")
 
 
 def gms_last_device_status(m: Manifest, stream=None) -> int:
