@@ -1,0 +1,190 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times (library
+defaults).  The oracle cannot redo 16-60 GB in seconds, so each test combines
+  * exact whole-output properties checked on the device with plain torch ops (every destination
+    byte equals its image byte, nothing else in the slab/pool changed, digest-in-place equals the
+    fused digest), with
+  * oracle values for sampled outputs: whole tensors where they are small enough (or ~1 GB once),
+    and individual 4 KiB blocks drawn from the large ones,
+  * host-made single-bit flips that gms_verify must name exactly.
+The mixed manifest (2.3 GB) is checked against the oracle in full, in both its 16-byte-rounded and
+raw odd-sized forms."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+from paper_2609_25451_b200 import gms  # noqa: E402
+from paper_2609_25451_b200 import workloads as W  # noqa: E402
+
+from gpu_harness import FILL, DeviceWorkload, oracle_record  # noqa: E402
+
+
+def u64(t):
+    return t.cpu().numpy().view(np.uint64)
+
+
+def expected_slab(w, image):
+    exp = torch.full((w.slab_bytes,), FILL, dtype=torch.uint8, device="cuda")
+    for r in w.rows:
+        s, d, n = int(r["src_offset"]), int(r["dst_offset"]), int(r["nbytes"])
+        exp[d:d + n] = image[s:s + n]
+    return exp
+
+
+def check_sampled_blocks(oracle, w, image, bd, base, rng, n_samples):
+    live = np.nonzero(w.rows["nbytes"] > 0)[0]
+    for _ in range(n_samples):
+        t = int(rng.choice(live))
+        n = int(w.rows[t]["nbytes"])
+        b = int(rng.integers(0, (n + 4095) // 4096))
+        if rng.random() < 0.2:
+            b = (n + 4095) // 4096 - 1  # favour ragged last blocks
+        lo, hi = b * 4096, min(n, b * 4096 + 4096)
+        s = int(w.rows[t]["src_offset"])
+        want = oracle.block_digest(image[s + lo:s + hi].cpu().numpy())
+        assert int(bd[int(base[t]) + b]) == want, (t, b)
+
+
+def test_llama3_8b_manifest_full_size(oracle):
+    w = W.llama3_8b_manifest()
+    image = torch.empty(w.image_bytes, dtype=torch.uint8, device="cuda")
+    W.fill_random_device(image, 991)
+    d = DeviceWorkload(w, image_dev=image)
+    bd, td = d.restore()
+    # every destination byte, every guard band
+    exp = expected_slab(w, image)
+    assert torch.equal(d.slab, exp)
+    del exp
+    # digest in place == fused digest (all 3.9 M blocks, all 291 tensors)
+    bd2, td2 = d.digest()
+    assert np.array_equal(bd, bd2) and np.array_equal(td, td2)
+    # oracle: every small tensor whole, one ~1 GB tensor whole, sampled blocks elsewhere
+    rec = oracle_record(oracle, w)
+    base, total = oracle.block_bases(rec)
+    assert total == bd.size == 3_921_026
+    rng = np.random.default_rng(17)
+    whole = [t for t in range(len(w.rows)) if int(w.rows[t]["nbytes"]) <= (16 << 20)][:80] + [0]
+    for t in whole:
+        s, n = int(w.rows[t]["src_offset"]), int(w.rows[t]["nbytes"])
+        T, obd = oracle.tensor_digest(image[s:s + n].cpu().numpy())
+        assert int(td[t]) == T, t
+        assert np.array_equal(bd[int(base[t]):int(base[t]) + obd.size], obd), t
+    check_sampled_blocks(oracle, w, image, bd, base, rng, 400)
+    # verify: clean, then 3 host-made single-bit flips
+    gms.gms_manifest_set_expected(d.m, d.bd_ptr())
+    assert d.verify(cap=8) == (0, [])
+    flips = W.flip_positions(w, 3, seed=23)
+    for row, byte, bit in flips:
+        d.flip(row, byte, bit)
+    bd3, td3 = d.digest()
+    count, pairs = d.verify(cap=8)
+    want = sorted(((row, byte // 4096) for row, byte, _ in flips))
+    assert count == 3 and pairs == [(int(w.rows[r]["tensor_id"]), b) for r, b in want]
+    changed = np.nonzero(bd3 != bd)[0].tolist()
+    assert changed == [int(base[r]) + b for r, b in want]
+    assert sorted(np.nonzero(td3 != td)[0].tolist()) == sorted({r for r, _ in want})
+    d.close()
+
+
+@pytest.mark.parametrize("round16", [True, False])
+def test_mixed_manifest_full_size_against_the_oracle_in_full(oracle, round16):
+    w = W.mixed_manifest(round16=round16)
+    image = torch.empty(w.image_bytes, dtype=torch.uint8, device="cuda")
+    W.fill_random_device(image, 992 + round16)
+    image_h = image.cpu().numpy()
+    slab_h = np.full(w.slab_bytes, FILL, np.uint8)
+    rc, obd, otd = oracle.restore(oracle_record(oracle, w), image_h, slab_h)
+    assert rc == 0
+    d = DeviceWorkload(w, image_dev=image)
+    bd, td = d.restore()
+    assert torch.equal(d.slab, torch.from_numpy(slab_h).cuda())
+    assert np.array_equal(bd, obd) and np.array_equal(td, otd)
+    bd2, td2 = d.digest()
+    assert np.array_equal(bd2, obd) and np.array_equal(td2, otd)
+    d.close()
+
+
+def test_kv_pool_full_size(oracle):
+    k = W.kv_pool_workload()
+    pool = torch.empty(k.pool_bytes, dtype=torch.uint8, device="cuda")
+    W.fill_random_device(pool, 993)
+    image = torch.empty(k.image_bytes, dtype=torch.uint8, device="cuda")
+    W.fill_random_device(image, 994)
+    kk = k.block_bytes // 4096
+    n_sel = len(k.ids)
+    # wrapping 64-bit sum of every pool block before the call (any changed bit changes the sum)
+    sums_before = pool.view(torch.int64).view(k.n_planes * k.n_blocks, -1).sum(dim=1)
+    ids = torch.from_numpy(k.ids).cuda()
+    bd = torch.zeros(n_sel * k.n_planes * kk, dtype=torch.int64, device="cuda")
+    kd = torch.zeros(n_sel, dtype=torch.int64, device="cuda")
+    st = torch.full((2,), -1, dtype=torch.int64, device="cuda")
+    desc = gms.KvPool(base=pool.data_ptr(), plane_stride=k.plane_stride, block_stride=k.block_stride, n_planes=k.n_planes,
+                      n_blocks=k.n_blocks, block_bytes=k.block_bytes)
+    gms.gms_kv_restore(desc, image, k.img_plane_stride, k.img_slot_stride, gms.SRC_DEVICE, ids, n_sel, bd, kd, st)
+    torch.cuda.synchronize()
+    assert st.tolist() == [0, 0]
+    pool3 = pool.view(k.n_planes, k.n_blocks, k.block_bytes)
+    img3 = image.view(k.n_planes, n_sel, k.block_bytes)
+    for p in range(k.n_planes):  # every selected block equals its image slot
+        assert torch.equal(pool3[p].index_select(0, ids.long()), img3[p]), p
+    sums_after = pool.view(torch.int64).view(k.n_planes * k.n_blocks, -1).sum(dim=1)
+    untouched = torch.ones(k.n_planes, k.n_blocks, dtype=torch.bool, device="cuda")
+    untouched[:, ids.long()] = False
+    assert torch.equal(sums_after.view(k.n_planes, k.n_blocks)[untouched], sums_before.view(k.n_planes, k.n_blocks)[untouched])
+    # oracle on sampled slots: all 64 planes of the slot, its 512 block digests and its KV-block digest
+    bd_h, kd_h = u64(bd).reshape(n_sel, k.n_planes, kk), u64(kd)
+    rng = np.random.default_rng(29)
+    for j in rng.choice(n_sel, size=40, replace=False).tolist() + [0, n_sel - 1]:
+        planes = img3[:, j, :].cpu().numpy()
+        T, obd = oracle.tensor_digest(planes.reshape(-1))
+        assert int(kd_h[j]) == T and np.array_equal(bd_h[j].reshape(-1), obd), j
+
+
+def test_host_sourced_70b_shard_full_size(oracle):
+    w = W.llama3_70b_tp8_shard_manifest(image_bytes=32 << 30)
+    try:
+        hptr, dview, arr = gms.gms_host_image_alloc(w.image_bytes)
+    except gms.GmsError as e:  # the box may not allow 32 GiB of pinned memory
+        pytest.skip(f"cannot pin 32 GiB of host memory here: {e}")
+    try:
+        cpu = torch.from_numpy(arr)
+        scratch = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+        for i, a in enumerate(range(0, w.image_bytes, 1 << 30)):
+            n = min(1 << 30, w.image_bytes - a)
+            W.fill_random_device(scratch[:n], 7000 + i)
+            cpu[a:a + n].copy_(scratch[:n])
+        del scratch
+        slab = torch.full((w.slab_bytes,), FILL, dtype=torch.uint8, device="cuda")
+        d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"), slab=slab)
+        bd, td = d.restore(image=dview, kind=gms.SRC_HOST_MAPPED)
+        # every destination byte against the host image (uploaded tensor by tensor), guards included
+        covered = torch.zeros(w.slab_bytes, dtype=torch.bool, device="cuda")
+        for r in w.rows:
+            s, dd, n = int(r["src_offset"]), int(r["dst_offset"]), int(r["nbytes"])
+            assert torch.equal(slab[dd:dd + n], cpu[s:s + n].cuda()), int(r["tensor_id"])
+            covered[dd:dd + n] = True
+        assert bool((slab[~covered] == FILL).all())
+        del covered
+        bd2, td2 = d.digest()
+        assert np.array_equal(bd, bd2) and np.array_equal(td, td2)
+        rec = oracle_record(oracle, w)
+        base, _ = oracle.block_bases(rec)
+        rng = np.random.default_rng(31)
+        small = [t for t in range(len(w.rows)) if int(w.rows[t]["nbytes"]) <= (4 << 20)]
+        for t in rng.choice(small, size=60, replace=False).tolist():
+            s, n = int(w.rows[t]["src_offset"]), int(w.rows[t]["nbytes"])
+            T, obd = oracle.tensor_digest(arr[s:s + n])
+            assert int(td[t]) == T and np.array_equal(bd[int(base[t]):int(base[t]) + obd.size], obd), t
+        live = np.nonzero(w.rows["nbytes"] > 0)[0]
+        for _ in range(300):
+            t = int(rng.choice(live))
+            n, s = int(w.rows[t]["nbytes"]), int(w.rows[t]["src_offset"])
+            b = int(rng.integers(0, (n + 4095) // 4096))
+            want = oracle.block_digest(arr[s + b * 4096:s + min(n, b * 4096 + 4096)])
+            assert int(bd[int(base[t]) + b]) == want, (t, b)
+        d.close()
+    finally:
+        torch.cuda.synchronize()
+        gms.gms_host_image_free(hptr)
