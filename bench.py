@@ -233,7 +233,7 @@ class KvBench:
         kk = k.block_bytes // 4096
         self.bd = torch.zeros(len(k.ids) * k.n_planes * kk, dtype=torch.int64, device=dev)
         self.kd = torch.zeros(len(k.ids), dtype=torch.int64, device=dev)
-        self.st = torch.zeros(2, dtype=torch.int64, device=dev)
+        self.st = torch.zeros(4, dtype=torch.int64, device=dev)
         self.desc = gms.KvPool(base=self.pool.data_ptr(), plane_stride=k.plane_stride, block_stride=k.block_stride,
                                n_planes=k.n_planes, n_blocks=k.n_blocks, block_bytes=k.block_bytes)
         self.payload = k.payload_bytes
@@ -250,7 +250,7 @@ class KvBench:
 
     def check(self):
         self.torch.cuda.synchronize()
-        assert self.st.tolist() == [0, 0]
+        assert self.st[:2].tolist() == [0, 0]
 
     def config(self):
         k = self.k

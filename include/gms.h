@@ -233,12 +233,13 @@ typedef struct {
  *                                            the slot's planes concatenated).
  * An id outside [0, n_blocks) is skipped: nothing is written to the pool, its
  * digests are 0, and d_status[0] counts it.  d_status[1] receives the device
- * status word.  Ids must be distinct (the caller's duty; duplicates race).
+ * status word; d_status[2..3] are scratch for the kernel's work counter.  Ids
+ * must be distinct (the caller's duty; duplicates race).
  *   image        (device-accessible) as for gms_restore; strides multiples of 16
  *   d_block_ids  (device) int32[n_sel]
  *   d_block_digests (device) n_sel*n_planes*k u64, may be NULL
  *   d_kv_digests (device) n_sel u64, may be NULL
- *   d_status     (device) 2 u64
+ *   d_status     (device) 4 u64
  * Errors: NULL, ALIGN, KIND, ARG, CUDA.
  */
 int gms_kv_restore(const gms_kv_pool *pool, const void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,

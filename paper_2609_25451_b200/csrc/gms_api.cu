@@ -153,7 +153,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         uint32_t total_warps = 148 * 12;
         if (!m->host_only) {
             gms::Geometry g;
-            cudaError_t e = gms::get_geometry(&g);
+            cudaError_t e = gms::get_geometry(gms::kRestore, &g);
             if (e != cudaSuccess) {
                 delete m;
                 return cuda_fail(e);
@@ -161,7 +161,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             total_warps = g.grid * g.warps;
             (void)cudaGetDevice(&m->device);
         }
-        uint32_t max_chunk = 16;
+        uint32_t max_chunk = 4;
         if (const char *v = getenv("GMS_CHUNK_BLOCKS")) {
             const long x = atol(v);
             if (x >= 1 && x <= (long)gms::kMaxChunkBlocks) max_chunk = (uint32_t)x;
@@ -179,7 +179,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             const size_t o_segoff = align_up(o_ids + n * sizeof(uint64_t), 256);
             const size_t o_segcnt = align_up(o_segoff + (size_t)m->n_segments * sizeof(uint64_t), 256);
             const size_t o_ctr = align_up(o_segcnt + (size_t)m->n_segments * sizeof(uint32_t), 256);
-            const size_t o_status = o_ctr + 128;
+            const size_t o_status = o_ctr + (size_t)gms::kMaxCounters * gms::kCounterStride * sizeof(unsigned int);
             const size_t total = o_status + 128;
             std::vector<uint8_t> h(total, 0);
             if (!m->chunks.empty()) memcpy(h.data() + o_chunks, m->chunks.data(), m->chunks.size() * sizeof(Chunk));
@@ -283,8 +283,11 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
     a.block_digests = d_block_digests;
     a.tensor_digests = d_tensor_digests;
     a.n_tensors = (uint32_t)m->entries.size();
-    a.work_counter = m->d_counter;
+    a.work_counters = m->d_counter;
     a.status = m->d_status;
+    a.hints = 0;
+    a.n_counters = 1;
+    a.group = 1;
     GMS_CUDA(store ? gms::launch_restore(a, static_cast<cudaStream_t>(stream))
                    : gms::launch_digest(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
@@ -379,6 +382,7 @@ int gms_kv_restore(const gms_kv_pool *pool, const void *image, uint64_t img_plan
     a.block_digests = d_block_digests;
     a.kv_digests = d_kv_digests;
     a.status = reinterpret_cast<unsigned long long *>(d_status);
+    a.hints = 0;
     GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
 }
@@ -414,7 +418,7 @@ int gms_host_image_free(void *host_ptr)
 int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *smem_bytes)
 {
     gms::Geometry g;
-    GMS_CUDA(gms::get_geometry(&g));
+    GMS_CUDA(gms::get_geometry(gms::kRestore, &g));
     if (grid_ctas) *grid_ctas = g.grid;
     if (warps_per_cta) *warps_per_cta = g.warps;
     if (smem_bytes) *smem_bytes = g.smem;

@@ -3,6 +3,8 @@
 #pragma once
 #include <cstddef>
 #include <cstdint>
+#include <cstdio>
+#include <cstdlib>
 #include <cuda_runtime.h>
 
 namespace gms {
@@ -10,6 +12,8 @@ namespace gms {
 constexpr uint32_t kBlockBytes = 4096;     // digest block
 constexpr uint32_t kMaxChunkBlocks = 32;   // one lane keeps one block digest of the chunk in flight
 constexpr uint64_t kG = 0x9E3779B97F4A7C15ull;
+constexpr uint32_t kMaxCounters = 32;      // work counters a manifest carries
+constexpr uint32_t kCounterStride = 64;    // 32-bit words between counters (256 B: separate L2 lines)
 
 // One unit of the persistent kernels' work list: a run of whole digest blocks of
 // one tensor (the last block of a tensor may be short).  32 bytes, read as 2 x 16 B.
@@ -29,8 +33,12 @@ struct Geometry {
     uint32_t warps;    // warps per CTA; every warp runs its own copy pipeline
     uint32_t stages;   // 4 KiB ring slots per warp
     uint32_t smem;     // dynamic shared memory per CTA
+    uint32_t hints;    // L2 eviction hints of the bulk copies: bits 0-1 loads, bits 2-3 stores (0 = none)
+    uint32_t counters; // work counters the chunk claims are spread over
+    uint32_t group;    // consecutive chunks bought by one claim
 };
-cudaError_t get_geometry(Geometry *g);
+enum Kind { kRestore = 0, kDigest = 1, kKv = 2 };  // the three streaming kernels have their own shapes
+cudaError_t get_geometry(Kind kind, Geometry *g);
 
 struct StreamArgs {
     const Chunk *chunks;
@@ -39,8 +47,11 @@ struct StreamArgs {
     uint64_t *block_digests;       // may be null
     uint64_t *tensor_digests;      // may be null
     uint32_t n_tensors;
-    unsigned int *work_counter;    // manifest-owned
+    unsigned int *work_counters;   // manifest-owned: kMaxCounters counters, kCounterStride words apart
     unsigned long long *status;    // manifest-owned device status word
+    uint32_t hints;                // filled in by the launcher
+    uint32_t n_counters;           // filled in by the launcher
+    uint32_t group;                // filled in by the launcher
 };
 
 struct KvArgs {
@@ -53,7 +64,8 @@ struct KvArgs {
     uint32_t n_sel;
     uint64_t *block_digests;       // may be null
     uint64_t *kv_digests;          // may be null
-    unsigned long long *status;    // [0] skipped ids, [1] device status word
+    unsigned long long *status;    // [0] skipped ids, [1] device status word, [2] work counter, [3] spare
+    uint32_t hints;                // filled in by the launcher
 };
 
 cudaError_t launch_restore(const StreamArgs &a, cudaStream_t s);

@@ -45,22 +45,13 @@ constexpr unsigned long long kDevTimeout = 1ull;     // GMS_DEV_TIMEOUT
 constexpr uint64_t kWaitLimitNs = 2000000000ull;     // 2 s per wait
 constexpr uint32_t kFull = 0xffffffffu;
 
-struct alignas(16) StageMeta {  // written by lane 0 when a block is issued, read by the warp when it lands
-    uint64_t dst;       // destination address of this block
-    uint32_t m;         // bytes of this block (1..4096)
-    uint32_t slot_last; // bits 0..7: index of the block in its chunk; bit 8: last block of the chunk
-    uint32_t gblock0;   // digest slot of the chunk's first block
-    uint32_t tblock0;   // tensor-relative index of the chunk's first block
-    uint32_t tensor;    // accumulator slot
-    uint32_t pad;
-};
-static_assert(sizeof(StageMeta) == 32, "StageMeta is 32 bytes");
-
 struct Item {  // one chunk as the pipeline sees it
     const uint8_t *src;
     uint8_t *dst;
     uint32_t nbytes, tensor, gblock0, tblock0;
 };
+
+constexpr uint32_t kFifo = 8;  // chunk records in flight between a warp's issue side and its digest side (>= ring slots)
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -149,44 +140,151 @@ __device__ __forceinline__ uint64_t warp_xor64(uint64_t v)
     return ((uint64_t)hi << 32) | lo;
 }
 
+// Bulk copies with an L2 eviction-priority hint (the payload is touched exactly once).
+__device__ __forceinline__ uint64_t l2_policy(uint32_t code)  // 1 evict_first, 2 evict_last, else evict_normal
+{
+    uint64_t pol;
+    if (code == 1)
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    else if (code == 2)
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    else
+        asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar, uint64_t pol)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                     dst_smem),
+                 "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar), "l"(pol)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store_hint(void *dst, uint32_t src_smem, uint32_t bytes, uint64_t pol)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(
+                     __cvta_generic_to_global(dst)),
+                 "r"(src_smem), "r"(bytes), "l"(pol)
+                 : "memory");
+}
+
 // ---------------------------------------------------------------- chunk providers (warp-uniform)
+// Both providers run one step ahead: the claim (an atomic) and the descriptor load for the chunk
+// after next are issued when a chunk is handed out and consumed a whole chunk later, so their
+// latency never sits between two blocks of a warp's pipeline.
 struct ListProvider {
     const Chunk *chunks;
     uint32_t n_chunks;
-    unsigned int *counter;
-    const uint8_t *image;  // null: digest in place (source = destination)
+    unsigned int *counters;  // n_counters work counters, kCounterStride words apart
+    uint32_t n_counters;
+    const uint8_t *image;    // null: digest in place (source = destination)
+    uint32_t home;           // the counter this warp is drawing from
+    uint32_t exhausted;      // counters found empty so far
+    uint32_t raw_next;       // lane 0: ticket drawn from counter `home` one step ahead
+    uint32_t group;          // consecutive chunks bought by one ticket
+    uint32_t grp_left, grp_idx;
+    uint4 da, db;            // buffered descriptor
+    bool have;
+
+    __device__ __forceinline__ void load(uint32_t idx)
+    {
+        const uint4 *p = reinterpret_cast<const uint4 *>(chunks + idx);
+        da = __ldg(p);
+        db = __ldg(p + 1);
+    }
+    __device__ __forceinline__ void draw(uint32_t lane)
+    {
+        if (lane == 0) raw_next = atomicAdd(counters + home * kCounterStride, 1u);
+    }
+    // Counter c hands out chunk runs c, c + n_counters, c + 2 n_counters, ... (a run = `group` consecutive chunks);
+    // warps are spread over the counters,
+    // so the chunks in flight stay a compact moving front of the work list while no single address takes all
+    // the atomics.  A warp whose counter has run dry moves on to the next one (that is the load balancing).
+    // The ticket used here was drawn one step earlier; the next one is drawn now and read a chunk later.
+    __device__ __forceinline__ bool advance(uint32_t lane, uint32_t &idx_out)
+    {
+        if (grp_left) {  // still inside the run of `group` consecutive chunks the last ticket bought
+            --grp_left;
+            idx_out = ++grp_idx;
+            return grp_idx < n_chunks;
+        }
+        for (;;) {
+            const uint32_t t = __shfl_sync(kFull, raw_next, 0);
+            const uint64_t idx = ((uint64_t)t * n_counters + home) * group;
+            if (idx < n_chunks) {
+                draw(lane);
+                idx_out = grp_idx = (uint32_t)idx;
+                grp_left = group - 1;
+                return true;
+            }
+            if (++exhausted >= n_counters) return false;
+            home = home + 1 == n_counters ? 0 : home + 1;
+            draw(lane);
+        }
+    }
+    __device__ __forceinline__ void init(uint32_t lane, uint32_t gwarp)
+    {
+        home = gwarp % n_counters;
+        exhausted = 0;
+        raw_next = 0;
+        grp_left = 0;
+        grp_idx = 0;
+        draw(lane);
+        uint32_t idx;
+        have = advance(lane, idx);
+        if (have) load(idx);
+    }
     __device__ __forceinline__ bool next(Item &it, uint32_t lane)
     {
-        uint32_t idx = 0;
-        if (lane == 0) idx = atomicAdd(counter, 1u);
-        idx = __shfl_sync(kFull, idx, 0);
-        if (idx >= n_chunks) return false;
-        const uint4 *p = reinterpret_cast<const uint4 *>(chunks + idx);
-        const uint4 a = __ldg(p), b = __ldg(p + 1);
-        const uint64_t src_off = ((uint64_t)a.y << 32) | a.x;
-        it.dst = reinterpret_cast<uint8_t *>(((uint64_t)a.w << 32) | a.z);
+        if (!have) return false;
+        const uint64_t src_off = ((uint64_t)da.y << 32) | da.x;
+        it.dst = reinterpret_cast<uint8_t *>(((uint64_t)da.w << 32) | da.z);
         it.src = image ? image + src_off : it.dst;
-        it.nbytes = b.x;
-        it.tensor = b.y;
-        it.gblock0 = b.z;
-        it.tblock0 = b.w;
+        it.nbytes = db.x;
+        it.tensor = db.y;
+        it.gblock0 = db.z;
+        it.tblock0 = db.w;
+        uint32_t idx;
+        have = advance(lane, idx);
+        if (have) load(idx);
         return true;
     }
 };
 
+// Units are (plane p, selected slot j), plane-major, so that consecutive units read consecutive
+// 32 KiB runs of the packed image.  Units are claimed in order from one counter (kept in the
+// caller's status array), one step ahead like the list provider, so the reads in flight form a
+// compact moving front of the image.
 struct KvProvider {
     KvArgs a;
-    uint64_t unit, stride, total;  // unit = j * n_planes + p
+    unsigned int *counter;
+    uint32_t total;     // n_planes * n_sel
+    uint32_t u_next;    // unit handed out next (already claimed)
+    int32_t id_next;    // its pool block id (already loaded)
+    uint32_t raw_next;  // lane 0: ticket for the unit after that
+
+    __device__ __forceinline__ void step(uint32_t lane)
+    {
+        u_next = __shfl_sync(kFull, raw_next, 0);
+        if (lane == 0) raw_next = atomicAdd(counter, 1u);
+        if (u_next < total) id_next = __ldg(a.ids + u_next % a.n_sel);
+    }
+    __device__ __forceinline__ void init(uint32_t lane)
+    {
+        raw_next = 0;
+        id_next = 0;
+        if (lane == 0) raw_next = atomicAdd(counter, 1u);
+        step(lane);
+    }
     __device__ __forceinline__ bool next(Item &it, uint32_t lane)
     {
         const uint32_t k = a.block_bytes >> 12;
-        while (unit < total) {
-            const uint32_t j = (uint32_t)(unit / a.n_planes), p = (uint32_t)(unit % a.n_planes);
-            const uint64_t u = unit;
-            unit += stride;
-            const int32_t id = __ldg(a.ids + j);
-            if (id < 0 || (uint32_t)id >= a.n_blocks) {  // skipped: digests 0, counted once per id
-                if (a.block_digests && lane < k) a.block_digests[u * k + lane] = 0;
+        while (u_next < total) {
+            const uint32_t p = u_next / a.n_sel, j = u_next % a.n_sel;
+            const int32_t id = id_next;
+            step(lane);
+            const uint32_t slot0 = (j * a.n_planes + p) * k;  // digest slots are laid out [j][p][block]
+            if (id < 0 || (uint32_t)id >= a.n_blocks) {       // skipped: digests 0, counted once per id
+                if (a.block_digests && lane < k) a.block_digests[(uint64_t)slot0 + lane] = 0;
                 if (p == 0 && lane == 0) atomicAdd(a.status, 1ull);
                 continue;
             }
@@ -194,7 +292,7 @@ struct KvProvider {
             it.dst = a.pool_base + (uint64_t)p * a.plane_stride + (uint64_t)id * a.block_stride;
             it.nbytes = a.block_bytes;
             it.tensor = j;
-            it.gblock0 = (uint32_t)(u * k);
+            it.gblock0 = slot0;
             it.tblock0 = p * k;
             return true;
         }
@@ -204,9 +302,10 @@ struct KvProvider {
 
 // ---------------------------------------------------------------- the per-warp pipeline
 template <int S, bool kStore, class Provider>
-__device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, StageMeta *meta, uint64_t *bars,
-                                             uint64_t *block_digests, uint64_t *accum, unsigned long long *status)
+__device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint4 *fifo, uint64_t *bars, uint64_t *block_digests,
+                                             uint64_t *accum, unsigned long long *status, uint32_t hints)
 {
+    static_assert(S <= (int)kFifo, "the chunk fifo must cover the ring");
     constexpr uint32_t LOOK = S - 1;  // blocks in flight ahead of the one being digested
     const uint32_t lane = threadIdx.x & 31u;
 
@@ -222,6 +321,8 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, Stag
         }
 
     const uint32_t ring_s = smem_u32(ring), bars_s = smem_u32(bars);
+    const uint32_t ld_hint = hints & 3u, st_hint = (hints >> 2) & 3u;
+    const uint64_t ld_pol = l2_policy(ld_hint), st_pol = l2_policy(st_hint);
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < S; ++s) mbar_init(bars_s + 8u * s, 1u);
@@ -229,11 +330,20 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, Stag
     }
     __syncwarp();
 
+    // issue-side cursor (the chunk being fetched) and digest-side cursor (the chunk being consumed);
+    // chunk records travel from one to the other through a small per-warp fifo in shared memory
     Item it{};
-    uint32_t it_blocks = 0, it_next = 0;
+    uint32_t it_blocks = 0, it_next = 0, chunks_in = 0;
+    uint64_t c_dst = 0;
+    uint32_t c_nbytes = 0, c_tensor = 0, c_gblock0 = 0, c_tblock0 = 0, c_blocks = 0, c_next = 0, chunks_out = 0;
     bool more = true, failed = false;
     uint32_t issued = 0, consumed = 0;
+    uint32_t is = 0;               // ring slot of the next block to issue   (issued % S)
+    uint32_t cs = 0, cparity = 0;  // ring slot and barrier phase of the next block to digest
     uint64_t myD = 0;
+    // share of a tensor digest gathered over consecutive chunks of the same tensor: one atomic per run, not per chunk
+    uint32_t run_tensor = 0xffffffffu;
+    uint64_t run_val = 0;
 
     for (;;) {
         // ---------------- issue: keep LOOK blocks ahead
@@ -243,8 +353,15 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, Stag
                 if (!more) break;
                 it_blocks = (it.nbytes + kBlockBytes - 1) >> 12;
                 it_next = 0;
+                if (lane == 0) {
+                    const uint64_t d = reinterpret_cast<uint64_t>(it.dst);
+                    fifo[2 * (chunks_in % kFifo)] = make_uint4((uint32_t)d, (uint32_t)(d >> 32), it.nbytes, it.tensor);
+                    fifo[2 * (chunks_in % kFifo) + 1] = make_uint4(it.gblock0, it.tblock0, 0u, 0u);
+                }
+                ++chunks_in;
             }
-            const uint32_t s = issued % S;
+            const uint32_t s = is;
+            is = (is + 1 == S) ? 0 : is + 1;
             const uint32_t off = it_next << 12;
             const uint32_t m = min(kBlockBytes, it.nbytes - off);
             const uint32_t m16 = m & ~15u;
@@ -266,64 +383,81 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, Stag
                 __syncwarp();
             }
             if (lane == 0) {
-                StageMeta md;
-                md.dst = reinterpret_cast<uint64_t>(it.dst + off);
-                md.m = m;
-                md.slot_last = it_next | ((it_next + 1 == it_blocks) ? 256u : 0u);
-                md.gblock0 = it.gblock0;
-                md.tblock0 = it.tblock0;
-                md.tensor = it.tensor;
-                md.pad = 0;
-                meta[s] = md;
                 mbar_arrive_expect_tx(bars_s + 8u * s, m16);
-                if (m16) bulk_load(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s);
+                if (m16) {
+                    if (ld_hint)
+                        bulk_load_hint(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s, ld_pol);
+                    else
+                        bulk_load(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s);
+                }
             }
             ++it_next;
             ++issued;
         }
         if (consumed == issued) break;
 
-        // ---------------- consume block `consumed`
-        const uint32_t s = consumed % S;
-        const bool ok = mbar_wait_bounded(bars_s + 8u * s, (consumed / S) & 1u);
+        // ---------------- digest block `consumed`
+        const uint32_t s = cs;
+        const bool ok = mbar_wait_bounded(bars_s + 8u * s, cparity);
+        if (++cs == S) cs = 0, cparity ^= 1u;
         if (!__all_sync(kFull, ok)) {
             failed = true;
             break;
         }
         __syncwarp();
-        const uint4 m0 = *reinterpret_cast<const uint4 *>(&meta[s]);
-        const uint4 m1 = *(reinterpret_cast<const uint4 *>(&meta[s]) + 1);
+        if (c_next == c_blocks) {  // next chunk record
+            const uint4 r0 = fifo[2 * (chunks_out % kFifo)], r1 = fifo[2 * (chunks_out % kFifo) + 1];
+            ++chunks_out;
+            c_dst = ((uint64_t)r0.y << 32) | r0.x;
+            c_nbytes = r0.z;
+            c_tensor = r0.w;
+            c_gblock0 = r1.x;
+            c_tblock0 = r1.y;
+            c_blocks = (c_nbytes + kBlockBytes - 1) >> 12;
+            c_next = 0;
+        }
         const uint8_t *stage = ring + s * kBlockBytes;
         if (kStore && lane == 0) {
-            const uint32_t m16 = m0.z & ~15u;
-            if (m16) bulk_store(reinterpret_cast<void *>(((uint64_t)m0.y << 32) | m0.x), ring_s + s * kBlockBytes, m16);
+            const uint32_t off = c_next << 12;
+            const uint32_t m16 = min(kBlockBytes, c_nbytes - off) & ~15u;
+            if (m16) {
+                if (st_hint)
+                    bulk_store_hint(reinterpret_cast<void *>(c_dst + off), ring_s + s * kBlockBytes, m16, st_pol);
+                else
+                    bulk_store(reinterpret_cast<void *>(c_dst + off), ring_s + s * kBlockBytes, m16);
+            }
             bulk_commit();
         }
         uint64_t acc = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint4 v = *reinterpret_cast<const uint4 *>(stage + 512 * j + 16 * lane);
-            acc ^= mix_head(((uint64_t)v.y << 32) | v.x, cfold[2 * j]);
-            acc ^= mix_head(((uint64_t)v.w << 32) | v.z, cfold[2 * j + 1]);
+            acc ^= mix_head(((uint64_t)v.y << 32) | v.x, cfold[2 * j]) ^ mix_head(((uint64_t)v.w << 32) | v.z, cfold[2 * j + 1]);
         }
         acc = warp_xor64(acc);
-        const uint64_t D = acc ^ (acc >> 31);
-        const uint32_t slot = m0.w & 255u;
-        if (lane == slot) myD = D;
-        if (m0.w & 256u) {  // chunk complete: block digests leave coalesced, one atomic for the tensor digest
-            const uint32_t gblock0 = m1.x, tblock0 = m1.y, tensor = m1.z;
+        if (lane == c_next) myD = acc ^ (acc >> 31);
+        ++c_next;
+        if (c_next == c_blocks) {  // chunk complete: block digests leave coalesced, one atomic for the tensor digest
             uint64_t t = 0;
-            if (lane <= slot) {
-                if (block_digests) block_digests[(uint64_t)gblock0 + lane] = myD;
-                t = mix_full(myD ^ ((uint64_t)(tblock0 + lane) * kG));
+            if (lane < c_blocks) {
+                if (block_digests) block_digests[(uint64_t)c_gblock0 + lane] = myD;
+                t = mix_full(myD ^ ((uint64_t)(c_tblock0 + lane) * kG));
             }
             t = warp_xor64(t);
-            if (lane == 0 && accum) atomicXor(reinterpret_cast<unsigned long long *>(accum + tensor), (unsigned long long)t);
+            if (c_tensor != run_tensor) {
+                if (run_tensor != 0xffffffffu && lane == 0 && accum)
+                    atomicXor(reinterpret_cast<unsigned long long *>(accum + run_tensor), (unsigned long long)run_val);
+                run_tensor = c_tensor;
+                run_val = 0;
+            }
+            run_val ^= t;
         }
         __syncwarp();  // every lane is done reading the slot before it is refilled
         ++consumed;
     }
 
+    if (run_tensor != 0xffffffffu && lane == 0 && accum)
+        atomicXor(reinterpret_cast<unsigned long long *>(accum + run_tensor), (unsigned long long)run_val);
     if (failed) {
         if (lane == 0) atomicOr(status, kDevTimeout);
         // bounded drain of what is still in flight into this warp's ring
@@ -334,18 +468,19 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, Stag
 
 struct SmemLayout {
     uint8_t *ring;
-    StageMeta *meta;
+    uint4 *fifo;
     uint64_t *bars;
 };
+constexpr uint32_t kWarpSmemExtra = kFifo * 32 + 8 * 8;  // fifo + up to 8 barriers
 template <int S>
 __device__ __forceinline__ SmemLayout carve(uint8_t *smem)
 {
     const uint32_t warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     SmemLayout l;
     l.ring = smem + (size_t)warp * S * kBlockBytes;
-    uint8_t *after = smem + (size_t)nwarps * S * kBlockBytes;
-    l.meta = reinterpret_cast<StageMeta *>(after) + warp * S;
-    l.bars = reinterpret_cast<uint64_t *>(after + (size_t)nwarps * S * sizeof(StageMeta)) + warp * S;
+    uint8_t *extra = smem + (size_t)nwarps * S * kBlockBytes + (size_t)warp * kWarpSmemExtra;
+    l.fifo = reinterpret_cast<uint4 *>(extra);
+    l.bars = reinterpret_cast<uint64_t *>(extra + kFifo * 32);
     return l;
 }
 
@@ -354,8 +489,15 @@ __global__ void __launch_bounds__(512, 1) gms_stream_kernel(StreamArgs a)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const SmemLayout l = carve<S>(smem);
-    ListProvider prov{a.chunks, a.n_chunks, a.work_counter, kStore ? a.image : nullptr};
-    run_pipeline<S, kStore>(prov, l.ring, l.meta, l.bars, a.block_digests, a.tensor_digests, a.status);
+    ListProvider prov;
+    prov.chunks = a.chunks;
+    prov.n_chunks = a.n_chunks;
+    prov.counters = a.work_counters;
+    prov.n_counters = a.n_counters;
+    prov.group = a.group;
+    prov.image = kStore ? a.image : nullptr;
+    prov.init(threadIdx.x & 31u, blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5));
+    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.hints);
 }
 
 template <int S>
@@ -363,53 +505,58 @@ __global__ void __launch_bounds__(512, 1) gms_kv_stream_kernel(KvArgs a)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const SmemLayout l = carve<S>(smem);
-    const uint32_t nwarps = blockDim.x >> 5;
-    KvProvider prov{a, (uint64_t)blockIdx.x * nwarps + (threadIdx.x >> 5), (uint64_t)gridDim.x * nwarps,
-                    (uint64_t)a.n_sel * a.n_planes};
-    run_pipeline<S, true>(prov, l.ring, l.meta, l.bars, a.block_digests, a.kv_digests, a.status + 1);
+    KvProvider prov;
+    prov.a = a;
+    prov.counter = reinterpret_cast<unsigned int *>(a.status + 2);
+    prov.total = a.n_sel * a.n_planes;
+    prov.init(threadIdx.x & 31u);
+    run_pipeline<S, true>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, a.hints);
 }
 
 // Clears the accumulators the streaming kernels XOR / add into.
-__global__ void gms_prologue_kernel(uint64_t *accum, uint64_t n_accum, unsigned int *counter, unsigned long long *status,
-                                    uint32_t n_status)
+__global__ void gms_prologue_kernel(uint64_t *accum, uint64_t n_accum, unsigned int *counters, uint32_t n_counters,
+                                    unsigned long long *status, uint32_t n_status)
 {
     const uint64_t i0 = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x, step = (uint64_t)gridDim.x * blockDim.x;
     if (accum)
         for (uint64_t i = i0; i < n_accum; i += step) accum[i] = 0;
-    if (i0 == 0 && counter) *counter = 0;
+    if (i0 < n_counters) counters[i0 * kCounterStride] = 0;
     if (i0 < n_status) status[i0] = 0;
 }
 
-uint32_t env_u32(const char *name, uint32_t dflt)
+// "w,s,c" from the environment (internal tuning hook), else the defaults
+void env_geom(const char *name, uint32_t &w, uint32_t &s, uint32_t &c)
 {
     const char *v = getenv(name);
-    if (!v || !*v) return dflt;
-    char *end = nullptr;
-    unsigned long x = strtoul(v, &end, 10);
-    return (end && *end == 0 && x > 0 && x < 1024) ? (uint32_t)x : dflt;
+    unsigned a = 0, b = 0, d = 0;
+    if (v && sscanf(v, "%u,%u,%u", &a, &b, &d) == 3 && a >= 1 && a <= 16 && (b == 3 || b == 4 || b == 6 || b == 8) && d >= 1 && d <= 4) {
+        w = a;
+        s = b;
+        c = d;
+    }
 }
 
 template <int S>
-cudaError_t set_attrs(uint32_t smem)
+cudaError_t set_attrs(Kind kind, uint32_t smem)
 {
-    cudaError_t e;
-    if ((e = cudaFuncSetAttribute(gms_stream_kernel<S, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    if ((e = cudaFuncSetAttribute(gms_stream_kernel<S, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    return cudaFuncSetAttribute(gms_kv_stream_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const void *f = kind == kRestore ? (const void *)gms_stream_kernel<S, true>
+                    : kind == kDigest ? (const void *)gms_stream_kernel<S, false>
+                                      : (const void *)gms_kv_stream_kernel<S>;
+    return cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
 constexpr int kMaxDevices = 64;
-Geometry g_geom[kMaxDevices];
-bool g_geom_ok[kMaxDevices];
+Geometry g_geom[kMaxDevices][3];
+bool g_geom_ok[kMaxDevices][3];
 
-cudaError_t prologue(uint64_t *accum, uint64_t n_accum, unsigned int *counter, unsigned long long *status, uint32_t n_status,
-                     cudaStream_t s)
+cudaError_t prologue(uint64_t *accum, uint64_t n_accum, unsigned int *counters, uint32_t n_counters, unsigned long long *status,
+                     uint32_t n_status, cudaStream_t s)
 {
     const uint32_t threads = 256;
     uint64_t blocks = accum ? (n_accum + threads - 1) / threads : 1;
     if (blocks < 1) blocks = 1;
     if (blocks > 1184) blocks = 1184;
-    gms_prologue_kernel<<<(uint32_t)blocks, threads, 0, s>>>(accum, n_accum, counter, status, n_status);
+    gms_prologue_kernel<<<(uint32_t)blocks, threads, 0, s>>>(accum, n_accum, counters, n_counters, status, n_status);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -418,15 +565,19 @@ template <bool kStore>
 cudaError_t launch_stream(const StreamArgs &a, cudaStream_t s)
 {
     Geometry g;
-    cudaError_t e = get_geometry(&g);
+    cudaError_t e = get_geometry(kStore ? kRestore : kDigest, &g);
     if (e) return e;
-    if ((e = prologue(a.tensor_digests, a.n_tensors, a.work_counter, a.status, 1, s))) return e;
+    if ((e = prologue(a.tensor_digests, a.n_tensors, a.work_counters, g.counters, a.status, 1, s))) return e;
     if (a.n_chunks == 0) return cudaSuccess;
+    StreamArgs b = a;
+    b.hints = g.hints;
+    b.n_counters = g.counters;
+    b.group = g.group;
     switch (g.stages) {
-    case 3: gms_stream_kernel<3, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
-    case 6: gms_stream_kernel<6, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
-    case 8: gms_stream_kernel<8, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
-    default: gms_stream_kernel<4, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
+    case 3: gms_stream_kernel<3, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
+    case 6: gms_stream_kernel<6, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
+    case 8: gms_stream_kernel<8, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
+    default: gms_stream_kernel<4, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
     }
     count_launches(1);
     return cudaGetLastError();
@@ -434,38 +585,55 @@ cudaError_t launch_stream(const StreamArgs &a, cudaStream_t s)
 
 }  // namespace
 
-cudaError_t get_geometry(Geometry *out)
+cudaError_t get_geometry(Kind kind, Geometry *out)
 {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!g_geom_ok[dev]) {
+    if (!g_geom_ok[dev][kind]) {
         int sms = 0, max_smem = 0;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev))) return e;
         if ((e = cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev))) return e;
         Geometry g;
-        // internal tuning hooks (defaults are what the benchmark numbers were taken with)
-        g.warps = env_u32("GMS_WARPS", 12);
-        g.stages = env_u32("GMS_STAGES", 4);
-        const uint32_t per_sm = env_u32("GMS_CTAS_PER_SM", 1);
-        if (g.stages != 3 && g.stages != 4 && g.stages != 6 && g.stages != 8) g.stages = 4;
-        if (g.warps > 16) g.warps = 16;
-        auto need = [&](uint32_t w) { return w * g.stages * (uint32_t)(kBlockBytes + sizeof(StageMeta) + 8); };
-        while (g.warps > 1 && need(g.warps) * per_sm > (uint32_t)max_smem) --g.warps;
+        uint32_t per_sm = 1;
+        // defaults are what the benchmark numbers were taken with
+        if (kind == kDigest) {
+            g.warps = 16, g.stages = 3;
+            env_geom("GMS_GEOM_DIGEST", g.warps, g.stages, per_sm);
+        } else if (kind == kRestore) {
+            g.warps = 8, g.stages = 6;
+            env_geom("GMS_GEOM_RESTORE", g.warps, g.stages, per_sm);
+        } else {
+            g.warps = 8, g.stages = 6;
+            env_geom("GMS_GEOM_KV", g.warps, g.stages, per_sm);
+        }
+        auto need = [&](uint32_t w) { return w * (g.stages * kBlockBytes + kWarpSmemExtra); };
+        while (g.warps > 1 && (need(g.warps) + 1024) * per_sm > (uint32_t)max_smem) --g.warps;
         g.smem = need(g.warps);
         g.grid = (uint32_t)sms * per_sm;
+        g.hints = 0;
+        if (const char *v = getenv("GMS_L2_HINTS")) g.hints = (uint32_t)atoi(v) & 15u;  // bits 0-1 load, 2-3 store
+        // claims: the restore kernels draw single chunks from one counter (strict list order keeps the bytes in
+        // flight a compact front, which HBM rewards); the digest kernel runs twice as fast per byte, so it
+        // spreads its claims over several counters and buys a run of chunks per ticket
+        g.counters = kind == kDigest ? 8 : 1;
+        g.group = kind == kDigest ? 4 : 1;
+        if (const char *v = getenv(kind == kDigest ? "GMS_CLAIM_DIGEST" : "GMS_CLAIM_RESTORE")) {
+            unsigned x = 0, y = 0;
+            if (sscanf(v, "%u,%u", &x, &y) == 2 && x >= 1 && x <= kMaxCounters && y >= 1 && y <= 64) g.counters = x, g.group = y;
+        }
         switch (g.stages) {
-        case 3: e = set_attrs<3>(g.smem); break;
-        case 6: e = set_attrs<6>(g.smem); break;
-        case 8: e = set_attrs<8>(g.smem); break;
-        default: e = set_attrs<4>(g.smem); break;
+        case 3: e = set_attrs<3>(kind, g.smem); break;
+        case 6: e = set_attrs<6>(kind, g.smem); break;
+        case 8: e = set_attrs<8>(kind, g.smem); break;
+        default: e = set_attrs<4>(kind, g.smem); break;
         }
         if (e) return e;
-        g_geom[dev] = g;
-        g_geom_ok[dev] = true;
+        g_geom[dev][kind] = g;
+        g_geom_ok[dev][kind] = true;
     }
-    *out = g_geom[dev];
+    *out = g_geom[dev][kind];
     return cudaSuccess;
 }
 
@@ -475,15 +643,17 @@ cudaError_t launch_digest(const StreamArgs &a, cudaStream_t s) { return launch_s
 cudaError_t launch_kv_restore(const KvArgs &a, cudaStream_t s)
 {
     Geometry g;
-    cudaError_t e = get_geometry(&g);
+    cudaError_t e = get_geometry(kKv, &g);
     if (e) return e;
-    if ((e = prologue(a.kv_digests, a.n_sel, nullptr, a.status, 2, s))) return e;
+    if ((e = prologue(a.kv_digests, a.n_sel, nullptr, 0, a.status, 4, s))) return e;
     if (a.n_sel == 0 || a.n_planes == 0) return cudaSuccess;
+    KvArgs b = a;
+    b.hints = g.hints;
     switch (g.stages) {
-    case 3: gms_kv_stream_kernel<3><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
-    case 6: gms_kv_stream_kernel<6><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
-    case 8: gms_kv_stream_kernel<8><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
-    default: gms_kv_stream_kernel<4><<<g.grid, g.warps * 32, g.smem, s>>>(a); break;
+    case 3: gms_kv_stream_kernel<3><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
+    case 6: gms_kv_stream_kernel<6><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
+    case 8: gms_kv_stream_kernel<8><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
+    default: gms_kv_stream_kernel<4><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
     }
     count_launches(1);
     return cudaGetLastError();

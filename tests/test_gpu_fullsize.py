@@ -119,12 +119,12 @@ def test_kv_pool_full_size(oracle):
     ids = torch.from_numpy(k.ids).cuda()
     bd = torch.zeros(n_sel * k.n_planes * kk, dtype=torch.int64, device="cuda")
     kd = torch.zeros(n_sel, dtype=torch.int64, device="cuda")
-    st = torch.full((2,), -1, dtype=torch.int64, device="cuda")
+    st = torch.full((4,), -1, dtype=torch.int64, device="cuda")
     desc = gms.KvPool(base=pool.data_ptr(), plane_stride=k.plane_stride, block_stride=k.block_stride, n_planes=k.n_planes,
                       n_blocks=k.n_blocks, block_bytes=k.block_bytes)
     gms.gms_kv_restore(desc, image, k.img_plane_stride, k.img_slot_stride, gms.SRC_DEVICE, ids, n_sel, bd, kd, st)
     torch.cuda.synchronize()
-    assert st.tolist() == [0, 0]
+    assert st[:2].tolist() == [0, 0]
     pool3 = pool.view(k.n_planes, k.n_blocks, k.block_bytes)
     img3 = image.view(k.n_planes, n_sel, k.block_bytes)
     for p in range(k.n_planes):  # every selected block equals its image slot

@@ -206,13 +206,13 @@ def run_kv(oracle, n_planes, n_blocks, block_bytes, ids, plane_gap, seed, host_m
         img = torch.from_numpy(img_h).cuda()
         img_ptr = img.data_ptr()
     ids_d = torch.from_numpy(np.ascontiguousarray(ids, dtype=np.int32)).cuda()
-    bd, kd, st = guarded_u64(n_sel * n_planes * k), guarded_u64(n_sel), guarded_u64(2)
+    bd, kd, st = guarded_u64(n_sel * n_planes * k), guarded_u64(n_sel), guarded_u64(4)
     desc = gms.KvPool(base=pool.data_ptr(), plane_stride=plane_stride, block_stride=block_bytes, n_planes=n_planes,
                       n_blocks=n_blocks, block_bytes=block_bytes)
     gms.gms_kv_restore(desc, img_ptr, ips, iss, gms.SRC_HOST_MAPPED if host_mapped else gms.SRC_DEVICE, ids_d, n_sel,
                        bd.data_ptr() + 8 * PAD, kd.data_ptr() + 8 * PAD, st.data_ptr() + 8 * PAD)
     torch.cuda.synchronize()
-    status = payload_of(st, 2)
+    status = payload_of(st, 4)
     assert int(status[0]) == oskip and int(status[1]) == 0
     assert np.array_equal(pool.cpu().numpy(), want_pool), "pool bytes differ"
     assert np.array_equal(payload_of(bd, n_sel * n_planes * k), obd)
