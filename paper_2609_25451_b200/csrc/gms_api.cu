@@ -161,13 +161,14 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             total_warps = g.grid * g.warps;
             (void)cudaGetDevice(&m->device);
         }
-        uint32_t max_chunk = 4;
-        if (const char *v = getenv("GMS_CHUNK_BLOCKS")) {
+        // Chunk length: 4 blocks (16 KiB).  Claims are made in strict list order, so short chunks keep all bytes in
+        // flight within a narrow moving window of the image, which HBM rewards; shorter than 4 and the per-chunk
+        // work shows.  Manifests too small to give every warp two such chunks are cut finer.
+        uint32_t chunk_blocks = (uint32_t)std::min<uint64_t>(4, std::max<uint64_t>(1, (n_blocks + 2ull * total_warps - 1) / (2ull * total_warps)));
+        if (const char *v = getenv("GMS_CHUNK_BLOCKS")) {  // internal tuning / test hook
             const long x = atol(v);
-            if (x >= 1 && x <= (long)gms::kMaxChunkBlocks) max_chunk = (uint32_t)x;
+            if (x >= 1 && x <= (long)gms::kMaxChunkBlocks) chunk_blocks = (uint32_t)x;
         }
-        const uint64_t want = n_blocks / (8ull * total_warps);
-        const uint32_t chunk_blocks = (uint32_t)std::min<uint64_t>(max_chunk, std::max<uint64_t>(1, want));
         build_chunks(*m, chunk_blocks);
         m->n_segments = (uint32_t)((n_blocks + gms::kVerifySegBlocks - 1) / gms::kVerifySegBlocks);
 

@@ -34,6 +34,8 @@
 // Every wait is bounded: a warp that does not see its own copy complete within
 // kWaitLimitNs sets GMS_DEV_TIMEOUT in the status word, drains (bounded) what
 // it has in flight and returns.
+#include <algorithm>
+
 #include "gms_internal.h"
 
 namespace gms {
@@ -572,7 +574,9 @@ cudaError_t launch_stream(const StreamArgs &a, cudaStream_t s)
     StreamArgs b = a;
     b.hints = g.hints;
     b.n_counters = g.counters;
-    b.group = g.group;
+    // a claim buys a run of chunks only while there are runs enough for every warp
+    b.group = (uint32_t)std::min<uint64_t>(g.group, std::max<uint64_t>(1, a.n_chunks / (4ull * g.grid * g.warps)));
+    if (b.group == 1 && a.n_chunks < 4ull * g.grid * g.warps) b.n_counters = std::min<uint32_t>(b.n_counters, 2);
     switch (g.stages) {
     case 3: gms_stream_kernel<3, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;
     case 6: gms_stream_kernel<6, kStore><<<g.grid, g.warps * 32, g.smem, s>>>(b); break;

@@ -111,6 +111,48 @@ __global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
     }
 }
 
+// Small inputs (a few thousand digest slots): the three passes in one CTA, one launch.
+constexpr uint32_t kSmallThreads = 1024;
+constexpr uint64_t kSmallBlocks = 16384;
+__global__ void __launch_bounds__(kSmallThreads) gms_verify_small_kernel(VerifyArgs a)
+{
+    __shared__ uint32_t warp_sum[kSmallThreads / 32];
+    const uint64_t per = (a.n_blocks + kSmallThreads - 1) / kSmallThreads;  // consecutive slots per thread
+    const uint64_t lo = (uint64_t)threadIdx.x * per, hi = lo + per < a.n_blocks ? lo + per : a.n_blocks;
+    uint32_t mine = 0;
+    for (uint64_t g = lo; g < hi; ++g) mine += a.computed[g] != a.expected[g];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
+        if ((int)lane >= d) incl += o;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    uint64_t rank = incl - mine, total = 0;
+    for (uint32_t w = 0; w < kSmallThreads / 32; ++w) {
+        if (w < warp) rank += warp_sum[w];
+        total += warp_sum[w];
+    }
+    if (threadIdx.x == 0) *a.count = total;
+    if (!mine) return;
+    Mismatch *out = static_cast<Mismatch *>(a.out);
+    for (uint64_t g = lo; g < hi; ++g) {
+        if (a.computed[g] == a.expected[g]) continue;
+        if (rank < a.cap) {
+            uint32_t l = 0, h = a.n_tensors;
+            while (h - l > 1) {
+                const uint32_t mid = l + (h - l) / 2;
+                if (a.block_base[mid] <= g) l = mid; else h = mid;
+            }
+            out[rank].tensor_id = a.tensor_ids[l];
+            out[rank].block = g - a.block_base[l];
+        }
+        ++rank;
+    }
+}
+
 __global__ void gms_copy_u64_kernel(uint64_t *dst, const uint64_t *src, uint64_t n)
 {
     const uint64_t step = (uint64_t)gridDim.x * blockDim.x;
@@ -124,6 +166,11 @@ cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
     if (a.n_segments == 0) {  // no digest slots at all: count = 0
         VerifyArgs z = a;
         gms_verify_scan_kernel<<<1, 32, 0, s>>>(z);
+        count_launches(1);
+        return cudaGetLastError();
+    }
+    if (a.n_blocks <= kSmallBlocks) {
+        gms_verify_small_kernel<<<1, kSmallThreads, 0, s>>>(a);
         count_launches(1);
         return cudaGetLastError();
     }

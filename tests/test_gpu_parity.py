@@ -132,8 +132,9 @@ def test_results_do_not_depend_on_entry_order_or_chunking(oracle, monkeypatch):
         d3.close()
 
 
-def test_many_mismatches_exceed_cap_in_order(oracle):
-    w = W.pack_layout("many", [4096 * 700 + 100, 4096 * 3000, 10, 4096 * 5000 + 1], seed=2)
+@pytest.mark.parametrize("scale", [1, 8])  # 8.7 K blocks: single-CTA verify; 70 K blocks: count / scan / emit
+def test_many_mismatches_exceed_cap_in_order(oracle, scale):
+    w = W.pack_layout("many", [4096 * 700 * scale + 100, 4096 * 3000 * scale, 10, 4096 * 5000 * scale + 1], seed=2)
     image = W.random_bytes_host(w.image_bytes, seed=10)
     rec = oracle_record(oracle, w)
     d = DeviceWorkload(w, image)
