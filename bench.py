@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["gms", "reference"], default="gms")
-    ap.add_argument("--workload", choices=["8b", "mixed", "tiny", "kv", "host70b"], default="8b")
+    ap.add_argument("--workload", choices=["8b", "mixed", "tiny", "kv", "host70b", "capture"], default="8b")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -217,6 +217,29 @@ class ManifestBench:
                 "step": "gms_digest + gms_verify + gms_restore(device image) + gms_verify",
                 "l2": "inputs larger than L2 (no flush)" if self.payload > (512 << 20) else "working set near L2 size; not flushed",
                 "payload_bytes": self.payload}
+
+
+class CaptureBench(ManifestBench):
+    """gms_capture of the 8B manifest (allocations -> packed device image, fused digest) + gms_verify."""
+
+    def __init__(self, torch, gms, W, dev):
+        super().__init__("8b", torch, gms, W, dev)
+        self.phase_names = ["capture", "verify"]
+        self.dominant, self.dominant_bytes = "capture", self.bytes_restore
+        self.traffic = self.bytes_restore + self.bytes_verify
+
+    def step(self, marks=None, image=None, kind=None):
+        g, m = self.gms, self.m
+        if marks: marks[0].record()
+        g.gms_capture(m, self.image, g.SRC_DEVICE, self.bd, self.td)
+        if marks: marks[1].record()
+        g.gms_verify(m, self.bd, self.mm, self.cap, self.cnt)
+        if marks: marks[2].record()
+
+    def config(self):
+        c = super().config()
+        c["step"] = "gms_capture(device image) + gms_verify"
+        return c
 
 
 class KvBench:
@@ -463,6 +486,8 @@ def main():
         bench = KvBench(torch, gms, W, dev)
     elif args.workload == "host70b":
         bench = None
+    elif args.workload == "capture":
+        bench = CaptureBench(torch, gms, W, dev)
     else:
         bench = ManifestBench(args.workload, torch, gms, W, dev)
 
@@ -511,7 +536,7 @@ def main():
         line["digest_frac_of_peak"] = line["digest_read_gbs"] / peak
 
     # ---- end to end: snapshot image in pinned host memory, verdict read back every step
-    if not args.no_e2e and isinstance(bench, ManifestBench):
+    if not args.no_e2e and type(bench) is ManifestBench:
         hptr, dview, cpu = host_image_of(torch, gms, bench.image)
         h2d_gbs = h2d_yardstick(torch, cpu, bench.image)
         pin_cnt = torch.zeros(1, dtype=torch.int64).pin_memory()
@@ -544,7 +569,7 @@ def main():
     elif not args.no_e2e:
         line["e2e"] = None
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and isinstance(bench, ManifestBench):
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and type(bench) is ManifestBench:
         line["cpu_baseline"] = cpu_baseline(args, bench, W, torch)
 
     if rank == 0:

@@ -157,6 +157,20 @@ int gms_restore(const gms_manifest *m, const void *image, uint32_t image_kind, u
                 uint64_t *d_tensor_digests, void *stream);
 
 /*
+ * gms_capture -- the inverse of gms_restore: Section 3.1, step 3 (device state is staged into a
+ * host-side image before it is serialised) and Section 3.2 (what is recorded at commit is what
+ * later reuse is checked against).  For every entry: image[src_offset, +nbytes) <- dst[0, nbytes),
+ * with D for each block and T for each tensor computed in the same pass -- the digests to hand to
+ * gms_manifest_set_expected.  `image` (device-accessible, written) is device memory or the device
+ * view of pinned mapped host memory, as `image_kind` says; bytes of the image that no entry covers
+ * are left alone.  Image ranges of different entries must not overlap (GMS_ERR_OVERLAP; restore
+ * allows shared sources, capture cannot).  Same kernel as gms_restore with the roles of source and
+ * destination exchanged.  Errors: NULL, ALIGN, KIND, OVERLAP, STATE, CUDA.
+ */
+int gms_capture(const gms_manifest *m, void *image, uint32_t image_kind, uint64_t *d_block_digests,
+                uint64_t *d_tensor_digests, void *stream);
+
+/*
  * gms_digest -- Section 3.2 (a replacement engine attaches surviving
  * allocations read-only) and Section 2.2 (reuse only if contents are intact).
  * Same outputs as gms_restore, computed over the destinations where they lie;
@@ -243,6 +257,16 @@ typedef struct {
  * Errors: NULL, ALIGN, KIND, ARG, CUDA.
  */
 int gms_kv_restore(const gms_kv_pool *pool, const void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
+                   uint32_t image_kind, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
+                   uint64_t *d_kv_digests, uint64_t *d_status, void *stream);
+
+/*
+ * gms_kv_capture -- the gather direction of the same extension (Section 6: committed KV blocks are
+ * kept in host memory or storage).  pool[p][d_block_ids[j]] is copied into slot j of the packed
+ * image for every plane p; arguments, digest layout, skipping of out-of-range ids (the slot is left
+ * alone) and status words are those of gms_kv_restore, with `image` written instead of read.
+ */
+int gms_kv_capture(const gms_kv_pool *pool, void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
                    uint32_t image_kind, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
                    uint64_t *d_kv_digests, uint64_t *d_status, void *stream);
 

@@ -157,6 +157,35 @@ int gmso_restore(const gmso_entry *e, size_t n, const uint8_t *image, uint64_t i
     return GMSO_OK;
 }
 
+/*
+ * Capture: the inverse of restore (Section 3.1, step 3: device state is staged into a host-side image before it
+ * is serialised; Section 3.2: what is captured at commit is what later reuse is checked against).  For each entry
+ * in record order the tensor's bytes are copied from its destination into the packed image at src_offset, and
+ * digested.  Image ranges must be pairwise disjoint here (two tensors packed onto the same image bytes would
+ * overwrite each other), which restore does not require.  Image bytes that no entry covers are left alone.
+ */
+int gmso_capture(const gmso_entry *e, size_t n, uint8_t *image, uint64_t image_bytes, const uint8_t *dst_base,
+                 uint64_t dst_bytes, uint64_t *block_digests, uint64_t *tensor_digests)
+{
+    int rc = gmso_validate(e, n, image_bytes, dst_bytes);
+    uint64_t base = 0;
+    if (rc) return rc;
+    if (n && (!image || !dst_base)) return GMSO_ERR_NULL;
+    for (size_t a = 0; a < n; ++a)
+        for (size_t b = a + 1; b < n; ++b)
+            if (e[a].nbytes && e[b].nbytes && e[a].src_offset < e[b].src_offset + e[b].nbytes &&
+                e[b].src_offset < e[a].src_offset + e[a].nbytes)
+                return GMSO_ERR_OVERLAP;
+    for (size_t t = 0; t < n; ++t) {
+        const uint8_t *src = dst_base + e[t].dst_offset;
+        if (e[t].nbytes) memcpy(image + e[t].src_offset, src, (size_t)e[t].nbytes);
+        uint64_t T = gmso_tensor_digest(image + e[t].src_offset, e[t].nbytes, block_digests ? block_digests + base : NULL);
+        if (tensor_digests) tensor_digests[t] = T;
+        base += gmso_num_blocks(e[t].nbytes);
+    }
+    return GMSO_OK;
+}
+
 /* Digest the destinations where they lie; nothing is written to them. */
 int gmso_digest(const gmso_entry *e, size_t n, const uint8_t *dst_base, uint64_t dst_bytes, uint64_t *block_digests,
                 uint64_t *tensor_digests)
@@ -227,6 +256,40 @@ int gmso_kv_restore(uint8_t *pool_base, uint64_t plane_stride, uint64_t block_st
             const uint8_t *src = image + (uint64_t)p * img_plane_stride + (uint64_t)j * img_slot_stride;
             uint8_t *dst = ok ? pool_base + (uint64_t)p * plane_stride + (uint64_t)ids[j] * block_stride : NULL;
             if (ok) memcpy(dst, src, block_bytes);
+            for (uint64_t c = 0; c < k; ++c) {
+                uint64_t q = (uint64_t)p * k + c;
+                uint64_t d = ok ? gmso_block_digest(dst + c * GMSO_BLOCK, GMSO_BLOCK) : 0;
+                if (block_digests) block_digests[((uint64_t)j * n_planes + p) * k + c] = d;
+                if (ok) K ^= gmso_mix(d ^ (q * GMSO_G));
+            }
+        }
+        if (kv_digests) kv_digests[j] = ok ? K : 0;
+    }
+    if (skipped) *skipped = skip;
+    return GMSO_OK;
+}
+
+/*
+ * Paged-KV subset capture: the gather direction of the same extension (committed KV blocks are kept outside the
+ * engine, Section 6).  Selected pool block ids[j] of every plane is copied into slot j of the packed image; digests
+ * are laid out exactly as in gmso_kv_restore.  An id outside [0, n_blocks) is skipped: its image slot is left
+ * alone, its digests are 0, and *skipped is incremented.
+ */
+int gmso_kv_capture(const uint8_t *pool_base, uint64_t plane_stride, uint64_t block_stride, uint32_t n_planes,
+                    uint32_t n_blocks, uint32_t block_bytes, uint8_t *image, uint64_t img_plane_stride,
+                    uint64_t img_slot_stride, const int32_t *ids, uint32_t n_sel, uint64_t *block_digests,
+                    uint64_t *kv_digests, uint64_t *skipped)
+{
+    uint64_t k = block_bytes / GMSO_BLOCK, skip = 0;
+    if (block_bytes == 0 || block_bytes % GMSO_BLOCK) return GMSO_ERR_ALIGN;
+    if (n_sel && (!pool_base || !image || !ids)) return GMSO_ERR_NULL;
+    for (uint32_t j = 0; j < n_sel; ++j) {
+        int ok = ids[j] >= 0 && (uint32_t)ids[j] < n_blocks;
+        uint64_t K = 0;
+        if (!ok) ++skip;
+        for (uint32_t p = 0; p < n_planes; ++p) {
+            uint8_t *dst = image + (uint64_t)p * img_plane_stride + (uint64_t)j * img_slot_stride;
+            if (ok) memcpy(dst, pool_base + (uint64_t)p * plane_stride + (uint64_t)ids[j] * block_stride, block_bytes);
             for (uint64_t c = 0; c < k; ++c) {
                 uint64_t q = (uint64_t)p * k + c;
                 uint64_t d = ok ? gmso_block_digest(dst + c * GMSO_BLOCK, GMSO_BLOCK) : 0;

@@ -61,6 +61,10 @@ def lib():
         L.gmso_block_bases.argtypes = [p, C.c_size_t, p]
         L.gmso_restore.restype = C.c_int
         L.gmso_restore.argtypes = [p, C.c_size_t, p, u64, p, u64, p, p]
+        L.gmso_capture.restype = C.c_int
+        L.gmso_capture.argtypes = [p, C.c_size_t, p, u64, p, u64, p, p]
+        L.gmso_kv_capture.restype = C.c_int
+        L.gmso_kv_capture.argtypes = [p, u64, u64, C.c_uint32, C.c_uint32, C.c_uint32, p, u64, u64, p, C.c_uint32, p, p, p]
         L.gmso_digest.restype = C.c_int
         L.gmso_digest.argtypes = [p, C.c_size_t, p, u64, p, p]
         L.gmso_verify.restype = u64
@@ -139,6 +143,20 @@ def restore(record: np.ndarray, image: np.ndarray, dst: np.ndarray):
     return int(rc), bd, td
 
 
+def capture(record: np.ndarray, image: np.ndarray, dst: np.ndarray):
+    """Gather the host slab ``dst`` into ``image`` (modified in place).
+
+    Returns (status, block_digests, tensor_digests).
+    """
+    record = np.ascontiguousarray(record, dtype=ENTRY_DTYPE)
+    img, d = image.view(np.uint8).reshape(-1), _bytes_view(dst)
+    assert img.flags.c_contiguous and img.flags.writeable
+    _, nb = block_bases(record)
+    bd, td = np.zeros(nb, dtype=np.uint64), np.zeros(len(record), dtype=np.uint64)
+    rc = lib().gmso_capture(_ptr(record), len(record), _ptr(img), img.size, _ptr(d), d.size, _ptr(bd), _ptr(td))
+    return int(rc), bd, td
+
+
 def digest(record: np.ndarray, dst: np.ndarray):
     """Digest the destinations in place.  Returns (status, block_digests, tensor_digests)."""
     record = np.ascontiguousarray(record, dtype=ENTRY_DTYPE)
@@ -174,6 +192,25 @@ def kv_restore(pool: np.ndarray, plane_stride: int, block_stride: int, n_planes:
     kd = np.zeros(len(ids), dtype=np.uint64)
     skipped = C.c_uint64(0)
     rc = lib().gmso_kv_restore(_ptr(pool_b), plane_stride, block_stride, n_planes, n_blocks, block_bytes, _ptr(img),
+                               img_plane_stride, img_slot_stride, _ptr(ids), len(ids), _ptr(bd), _ptr(kd),
+                               C.addressof(skipped))
+    return int(rc), bd, kd, int(skipped.value)
+
+
+def kv_capture(pool: np.ndarray, plane_stride: int, block_stride: int, n_planes: int, n_blocks: int,
+               block_bytes: int, image: np.ndarray, img_plane_stride: int, img_slot_stride: int, ids: np.ndarray):
+    """Gather selected pool blocks into the host image (modified in place).
+
+    Returns (status, block_digests, kv_digests, skipped).
+    """
+    pool_b = _bytes_view(pool)
+    img = image.view(np.uint8).reshape(-1)
+    ids = np.ascontiguousarray(ids, dtype=np.int32)
+    k = block_bytes // BLOCK
+    bd = np.zeros(len(ids) * n_planes * k, dtype=np.uint64)
+    kd = np.zeros(len(ids), dtype=np.uint64)
+    skipped = C.c_uint64(0)
+    rc = lib().gmso_kv_capture(_ptr(pool_b), plane_stride, block_stride, n_planes, n_blocks, block_bytes, _ptr(img),
                                img_plane_stride, img_slot_stride, _ptr(ids), len(ids), _ptr(bd), _ptr(kd),
                                C.addressof(skipped))
     return int(rc), bd, kd, int(skipped.value)

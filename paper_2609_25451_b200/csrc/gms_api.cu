@@ -22,6 +22,7 @@ struct gms_manifest {
     std::vector<Chunk> chunks;
     uint64_t image_bytes = 0, payload = 0, n_blocks = 0;
     bool host_only = false;
+    bool sources_disjoint = true;  // image ranges pairwise disjoint (needed by gms_capture only)
     int device = -1;
     // device tables (one allocation) and the recorded digests (allocated on first use)
     uint8_t *d_tables = nullptr;
@@ -135,7 +136,13 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             if (reinterpret_cast<uint64_t>(p.dst) + p.nbytes > reinterpret_cast<uint64_t>(q.dst)) return GMS_ERR_OVERLAP;
         }
 
+        bool sources_disjoint = true;
+        std::sort(live.begin(), live.end(), [&](uint32_t a, uint32_t b) { return entries[a].src_offset < entries[b].src_offset; });
+        for (size_t i = 1; i < live.size(); ++i)
+            if (entries[live[i - 1]].src_offset + entries[live[i - 1]].nbytes > entries[live[i]].src_offset) sources_disjoint = false;
+
         gms_manifest *m = new gms_manifest();
+        m->sources_disjoint = sources_disjoint;
         m->entries.assign(entries, entries + n);
         m->image_bytes = image_bytes;
         m->payload = payload;
@@ -275,7 +282,7 @@ int gms_manifest_set_expected(gms_manifest *m, const uint64_t *d_block_digests, 
 }
 
 static int stream_call(const gms_manifest *m, const void *image, bool store, uint64_t *d_block_digests,
-                       uint64_t *d_tensor_digests, void *stream)
+                       uint64_t *d_tensor_digests, void *stream, bool capture = false)
 {
     gms::StreamArgs a;
     a.chunks = m->d_chunks;
@@ -289,6 +296,7 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
     a.hints = 0;
     a.n_counters = 1;
     a.group = 1;
+    a.capture = capture ? 1u : 0u;
     GMS_CUDA(store ? gms::launch_restore(a, static_cast<cudaStream_t>(stream))
                    : gms::launch_digest(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
@@ -306,6 +314,21 @@ int gms_restore(const gms_manifest *m, const void *image, uint32_t image_kind, u
         if (rc) return rc;
     }
     return stream_call(m, image, true, d_block_digests, d_tensor_digests, stream);
+}
+
+int gms_capture(const gms_manifest *m, void *image, uint32_t image_kind, uint64_t *d_block_digests,
+                uint64_t *d_tensor_digests, void *stream)
+{
+    if (!m || (!image && m->payload)) return GMS_ERR_NULL;
+    if (image_kind != GMS_SRC_DEVICE && image_kind != GMS_SRC_HOST_MAPPED) return GMS_ERR_KIND;
+    if (reinterpret_cast<uint64_t>(image) & 15u) return GMS_ERR_ALIGN;
+    if (!m->sources_disjoint) return GMS_ERR_OVERLAP;
+    if (m->host_only) return GMS_ERR_STATE;
+    if (image) {
+        const int rc = check_kind(image, image_kind);
+        if (rc) return rc;
+    }
+    return stream_call(m, image, true, d_block_digests, d_tensor_digests, stream, true);
 }
 
 int gms_digest(const gms_manifest *m, uint64_t *d_block_digests, uint64_t *d_tensor_digests, void *stream)
@@ -348,9 +371,9 @@ int gms_last_device_status(const gms_manifest *m, void *stream, uint64_t *word)
     return (w & GMS_DEV_TIMEOUT) ? GMS_ERR_TIMEOUT : GMS_OK;
 }
 
-int gms_kv_restore(const gms_kv_pool *pool, const void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
+static int kv_call(const gms_kv_pool *pool, const void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
                    uint32_t image_kind, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
-                   uint64_t *d_kv_digests, uint64_t *d_status, void *stream)
+                   uint64_t *d_kv_digests, uint64_t *d_status, void *stream, bool capture)
 {
     if (!pool || !d_status) return GMS_ERR_NULL;
     if (image_kind != GMS_SRC_DEVICE && image_kind != GMS_SRC_HOST_MAPPED) return GMS_ERR_KIND;
@@ -384,8 +407,25 @@ int gms_kv_restore(const gms_kv_pool *pool, const void *image, uint64_t img_plan
     a.kv_digests = d_kv_digests;
     a.status = reinterpret_cast<unsigned long long *>(d_status);
     a.hints = 0;
+    a.capture = capture ? 1u : 0u;
     GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
+}
+
+int gms_kv_restore(const gms_kv_pool *pool, const void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
+                   uint32_t image_kind, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
+                   uint64_t *d_kv_digests, uint64_t *d_status, void *stream)
+{
+    return kv_call(pool, image, img_plane_stride, img_slot_stride, image_kind, d_block_ids, n_sel, d_block_digests, d_kv_digests,
+                   d_status, stream, false);
+}
+
+int gms_kv_capture(const gms_kv_pool *pool, void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
+                   uint32_t image_kind, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
+                   uint64_t *d_kv_digests, uint64_t *d_status, void *stream)
+{
+    return kv_call(pool, image, img_plane_stride, img_slot_stride, image_kind, d_block_ids, n_sel, d_block_digests, d_kv_digests,
+                   d_status, stream, true);
 }
 
 int gms_host_image_alloc(uint64_t nbytes, void **host_ptr, void **device_view)

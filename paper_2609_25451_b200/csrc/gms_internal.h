@@ -52,6 +52,7 @@ struct StreamArgs {
     uint32_t hints;                // filled in by the launcher
     uint32_t n_counters;           // filled in by the launcher
     uint32_t group;                // filled in by the launcher
+    uint32_t capture;              // 1: gather allocations into the image (restore kernel with roles swapped)
 };
 
 struct KvArgs {
@@ -65,6 +66,7 @@ struct KvArgs {
     uint64_t *block_digests;       // may be null
     uint64_t *kv_digests;          // may be null
     unsigned long long *status;    // [0] skipped ids, [1] device status word, [2] work counter, [3] spare
+    uint32_t capture;              // 1: gather pool blocks into the image
     uint32_t hints;                // filled in by the launcher
 };
 

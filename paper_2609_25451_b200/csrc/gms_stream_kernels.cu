@@ -179,6 +179,7 @@ struct ListProvider {
     unsigned int *counters;  // n_counters work counters, kCounterStride words apart
     uint32_t n_counters;
     const uint8_t *image;    // null: digest in place (source = destination)
+    bool capture;            // copy allocation -> image instead of image -> allocation
     uint32_t home;           // the counter this warp is drawing from
     uint32_t exhausted;      // counters found empty so far
     uint32_t raw_next;       // lane 0: ticket drawn from counter `home` one step ahead
@@ -241,6 +242,11 @@ struct ListProvider {
         const uint64_t src_off = ((uint64_t)da.y << 32) | da.x;
         it.dst = reinterpret_cast<uint8_t *>(((uint64_t)da.w << 32) | da.z);
         it.src = image ? image + src_off : it.dst;
+        if (capture) {  // gather: the allocation is the source, the packed image the destination
+            const uint8_t *alloc = it.dst;
+            it.dst = const_cast<uint8_t *>(it.src);
+            it.src = alloc;
+        }
         it.nbytes = db.x;
         it.tensor = db.y;
         it.gblock0 = db.z;
@@ -290,8 +296,10 @@ struct KvProvider {
                 if (p == 0 && lane == 0) atomicAdd(a.status, 1ull);
                 continue;
             }
-            it.src = a.image + (uint64_t)p * a.img_plane_stride + (uint64_t)j * a.img_slot_stride;
-            it.dst = a.pool_base + (uint64_t)p * a.plane_stride + (uint64_t)id * a.block_stride;
+            uint8_t *img = const_cast<uint8_t *>(a.image) + (uint64_t)p * a.img_plane_stride + (uint64_t)j * a.img_slot_stride;
+            uint8_t *blk = a.pool_base + (uint64_t)p * a.plane_stride + (uint64_t)id * a.block_stride;
+            it.src = a.capture ? blk : img;
+            it.dst = a.capture ? img : blk;
             it.nbytes = a.block_bytes;
             it.tensor = j;
             it.gblock0 = slot0;
@@ -498,6 +506,7 @@ __global__ void __launch_bounds__(512, 1) gms_stream_kernel(StreamArgs a)
     prov.n_counters = a.n_counters;
     prov.group = a.group;
     prov.image = kStore ? a.image : nullptr;
+    prov.capture = kStore && a.capture;
     prov.init(threadIdx.x & 31u, blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5));
     run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.hints);
 }

@@ -30,8 +30,8 @@ MISMATCH_DTYPE = np.dtype([("tensor_id", "<u8"), ("block", "<u8")])
 
 EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
-    "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_digest",
-    "gms_verify", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_host_image_alloc", "gms_host_image_free",
+    "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
+    "gms_verify", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_host_image_alloc", "gms_host_image_free",
     "gms_launch_geometry", "gms_kernel_launches", "gms_set_device", "gms_strerror", "gms_last_cuda_error", "gms_version",
 )
 
@@ -72,11 +72,13 @@ def lib():
             "gms_manifest_chunk": (i, [p, u64, pu64, pu64, pu64]),
             "gms_manifest_set_expected": (i, [p, p, p]),
             "gms_restore": (i, [p, p, u32, p, p, p]),
+            "gms_capture": (i, [p, p, u32, p, p, p]),
             "gms_digest": (i, [p, p, p, p]),
             "gms_verify": (i, [p, p, p, u32, p, p]),
             "gms_verify_flat_noalloc": (i, [p, p, u64, u64, p, u32, p, p]),
             "gms_last_device_status": (i, [p, p, pu64]),
             "gms_kv_restore": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
+            "gms_kv_capture": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
             "gms_host_image_alloc": (i, [u64, pp, pp]),
             "gms_host_image_free": (i, [p]),
             "gms_launch_geometry": (i, [pu32, pu32, pu32]),
@@ -177,6 +179,11 @@ def gms_restore(m: Manifest, image, image_kind: int, d_block_digests, d_tensor_d
                              _stream(stream)), "gms_restore")
 
 
+def gms_capture(m: Manifest, image, image_kind: int, d_block_digests, d_tensor_digests, stream=None):
+    _check(lib().gms_capture(m.handle, _dev(image), image_kind, _dev(d_block_digests), _dev(d_tensor_digests),
+                             _stream(stream)), "gms_capture")
+
+
 def gms_digest(m: Manifest, d_block_digests, d_tensor_digests, stream=None):
     _check(lib().gms_digest(m.handle, _dev(d_block_digests), _dev(d_tensor_digests), _stream(stream)), "gms_digest")
 
@@ -202,6 +209,13 @@ def gms_kv_restore(pool: KvPool, image, img_plane_stride: int, img_slot_stride: 
     _check(lib().gms_kv_restore(C.byref(pool), _dev(image), img_plane_stride, img_slot_stride, image_kind,
                                 _dev(d_block_ids), n_sel, _dev(d_block_digests), _dev(d_kv_digests), _dev(d_status),
                                 _stream(stream)), "gms_kv_restore")
+
+
+def gms_kv_capture(pool: KvPool, image, img_plane_stride: int, img_slot_stride: int, image_kind: int, d_block_ids,
+                   n_sel: int, d_block_digests, d_kv_digests, d_status, stream=None):
+    _check(lib().gms_kv_capture(C.byref(pool), _dev(image), img_plane_stride, img_slot_stride, image_kind,
+                                _dev(d_block_ids), n_sel, _dev(d_block_digests), _dev(d_kv_digests), _dev(d_status),
+                                _stream(stream)), "gms_kv_capture")
 
 
 def gms_host_image_alloc(nbytes: int):

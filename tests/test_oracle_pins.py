@@ -330,3 +330,58 @@ def test_kv_restore_reduces_to_restore_and_tensor_digest(oracle):
         T, _ = oracle.tensor_digest(np.concatenate(cat))
         assert int(kd[j]) == (T if ok else 0)
     assert np.array_equal(pool, want_pool)
+
+
+def test_capture_is_the_inverse_of_restore(oracle):
+    rng = np.random.default_rng(51)
+    rows, image_bytes, slab_bytes = _random_record(rng, 35, 15000)
+    rec = oracle.make_record(rows)
+    slab = rng.integers(0, 256, slab_bytes, dtype=np.uint8)
+    image = np.full(image_bytes, 0xC3, np.uint8)
+    rc, bd, td = oracle.capture(rec, image, slab)
+    assert rc == 0
+    covered = np.zeros(image_bytes, bool)
+    for tid, so, do, nb in rows:
+        assert np.array_equal(image[so : so + nb], slab[do : do + nb])  # brute-force byte compare
+        covered[so : so + nb] = True
+    assert np.all(image[~covered] == 0xC3)  # image bytes no entry covers are left alone
+    # the digests of a capture are the digests of the destinations where they lie ...
+    rc2, bd2, td2 = oracle.digest(rec, slab)
+    assert np.array_equal(bd, bd2) and np.array_equal(td, td2)
+    # ... and restoring the captured image gives back the same bytes and the same digests
+    slab2 = np.zeros(slab_bytes, np.uint8)
+    rc3, bd3, td3 = oracle.restore(rec, image, slab2)
+    assert rc3 == 0 and np.array_equal(bd3, bd) and np.array_equal(td3, td)
+    for tid, so, do, nb in rows:
+        assert np.array_equal(slab2[do : do + nb], slab[do : do + nb])
+    # two tensors packed onto the same image bytes are refused by capture (restore accepts shared sources)
+    shared = oracle.make_record([(1, 0, 0, 100), (2, 0, 112, 100)])
+    assert oracle.validate(shared, 1000, 1000) == oracle.OK
+    assert oracle.capture(shared, np.zeros(1000, np.uint8), np.zeros(1000, np.uint8))[0] == oracle.ERR_OVERLAP
+
+
+def test_kv_capture_is_the_inverse_of_kv_restore(oracle):
+    rng = np.random.default_rng(52)
+    n_planes, n_blocks, bb = 5, 13, 8192
+    ids = np.array([3, 12, -2, 0, 13, 7], np.int32)  # -2 and 13 are out of range
+    plane_stride, ips = n_blocks * bb + 512, len(ids) * bb
+    pool = rng.integers(0, 256, n_planes * plane_stride, dtype=np.uint8)
+    image = np.full(n_planes * ips, 0x77, np.uint8)
+    rc, bd, kd, skipped = oracle.kv_capture(pool, plane_stride, bb, n_planes, n_blocks, bb, image, ips, bb, ids)
+    assert rc == 0 and skipped == 2
+    for j, blk in enumerate(ids):
+        for p in range(n_planes):
+            slot = image[p * ips + j * bb :][:bb]
+            if 0 <= blk < n_blocks:
+                assert np.array_equal(slot, pool[p * plane_stride + blk * bb :][:bb])
+            else:
+                assert np.all(slot == 0x77)
+    # scattering the captured image back reproduces the pool and the same digests
+    pool2 = pool.copy()
+    for j, blk in enumerate(ids):
+        if 0 <= blk < n_blocks:
+            for p in range(n_planes):
+                pool2[p * plane_stride + blk * bb :][:bb] = 0
+    rc2, bd2, kd2, skipped2 = oracle.kv_restore(pool2, plane_stride, bb, n_planes, n_blocks, bb, image, ips, bb, ids)
+    assert rc2 == 0 and skipped2 == 2 and np.array_equal(pool2, pool)
+    assert np.array_equal(bd2, bd) and np.array_equal(kd2, kd)
