@@ -76,6 +76,7 @@ extern "C" {
 #define GMS_ERR_STATE (-10)   /* manifest has no device tables / no recorded digests          */
 #define GMS_ERR_ARG (-11)     /* an argument is out of its documented range                   */
 #define GMS_ERR_TOO_LARGE (-12) /* more digest blocks than gms_verify_flat_noalloc has room for */
+#define GMS_ERR_IO (-13)      /* a file read failed or the file is shorter than the image     */
 
 /* where the packed snapshot image lives */
 #define GMS_SRC_DEVICE 0u      /* device memory (a staging buffer in HBM)                     */
@@ -277,6 +278,31 @@ int gms_kv_capture(const gms_kv_pool *pool, void *image, uint64_t img_plane_stri
  */
 int gms_host_image_alloc(uint64_t nbytes, void **host_ptr, void **device_view);
 int gms_host_image_free(void *host_ptr);
+
+/*
+ * gms_pipe_* / gms_restore_fd -- Section 4, GMS paragraph: with a cold service, a read-write client
+ * repopulates model state from storage while the process is being restored; Section 3.1 prices it
+ * at S / B_eff.  The image is read from a file descriptor, never resident as a whole: a ring of
+ * `n_buffers` pinned, device-mapped buffers of `buffer_bytes` each (>= 1 MiB, multiple of 4096) is
+ * filled by `n_readers` threads with pread(), and each filled buffer is consumed by the restore
+ * kernel (which reads it across the host link, scatters and digests) while the next one is read.
+ * gms_restore_fd is synchronous: on return the stream has been synchronised and the outputs hold
+ * exactly what gms_restore would have produced from the same bytes (image byte k = file byte
+ * file_offset + k).  One restore at a time per pipe.  Errors: NULL, ARG (bad sizes; a chunk larger
+ * than a buffer), NOMEM, STATE, IO (read error or file shorter than the image), CUDA.
+ */
+typedef struct gms_pipe gms_pipe; /* opaque */
+typedef struct {
+    uint64_t windows;          /* buffers' worth of image consumed                          */
+    uint64_t bytes_read;       /* bytes read from the file                                  */
+    double wait_read_seconds;  /* host time spent waiting for readers (storage-bound share) */
+    double wait_gpu_seconds;   /* host time spent waiting for a buffer to be released       */
+    double total_seconds;      /* wall time of the call                                     */
+} gms_pipe_stats;
+int gms_pipe_create(uint32_t n_buffers, uint64_t buffer_bytes, uint32_t n_readers, gms_pipe **out);
+int gms_pipe_destroy(gms_pipe *p);
+int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_offset, uint64_t *d_block_digests,
+                   uint64_t *d_tensor_digests, void *stream, gms_pipe_stats *stats);
 
 /* Launch geometry of the streaming kernels on the current device (for reporting). */
 int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *smem_bytes);

@@ -6,6 +6,7 @@
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <numeric>
 #include <string>
@@ -34,6 +35,10 @@ struct gms_manifest {
     uint64_t *d_expected = nullptr;
     bool has_expected = false;
     uint32_t n_segments = 0;
+    // chunk list sorted by source offset, for restores fed window by window (built on first use)
+    mutable std::mutex mu;
+    mutable std::vector<Chunk> by_src;
+    mutable Chunk *d_by_src = nullptr;
 };
 
 namespace {
@@ -95,6 +100,69 @@ int check_kind(const void *image, uint32_t kind)
 namespace gms {
 void count_launches(uint32_t n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 int report_cuda_error(cudaError_t e) { return cuda_fail(e); }
+}  // namespace gms
+
+namespace gms {
+
+uint64_t manifest_n_tensors(const gms_manifest *m) { return m->entries.size(); }
+
+int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vector<SrcWindow> *out)
+{
+    if (m->host_only) return GMS_ERR_STATE;
+    std::lock_guard<std::mutex> lock(m->mu);
+    if (m->by_src.empty() && !m->chunks.empty()) {
+        m->by_src = m->chunks;
+        std::stable_sort(m->by_src.begin(), m->by_src.end(), [](const Chunk &a, const Chunk &b) { return a.src_off < b.src_off; });
+        cudaError_t e = cudaMalloc(&m->d_by_src, m->by_src.size() * sizeof(Chunk));
+        if (e != cudaSuccess) {
+            m->by_src.clear();
+            (void)cudaGetLastError();
+            return e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : cuda_fail(e);
+        }
+        e = cudaMemcpy(m->d_by_src, m->by_src.data(), m->by_src.size() * sizeof(Chunk), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    out->clear();
+    size_t i = 0;
+    while (i < m->by_src.size()) {
+        SrcWindow w;
+        w.first_chunk = (uint32_t)i;
+        w.src_lo = m->by_src[i].src_off;
+        w.src_hi = w.src_lo;
+        while (i < m->by_src.size()) {
+            const uint64_t end = m->by_src[i].src_off + m->by_src[i].nbytes;
+            if (std::max(end, w.src_hi) - w.src_lo > buffer_bytes) break;
+            w.src_hi = std::max(end, w.src_hi);
+            ++i;
+        }
+        if (i == w.first_chunk) return GMS_ERR_ARG;  // a single chunk does not fit the buffer
+        w.n_chunks = (uint32_t)(i - w.first_chunk);
+        out->push_back(w);
+    }
+    return GMS_OK;
+}
+
+int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void *window_base, bool first,
+                           uint64_t *d_block_digests, uint64_t *d_tensor_digests, cudaStream_t s)
+{
+    StreamArgs a;
+    a.chunks = m->d_by_src + w.first_chunk;
+    a.n_chunks = w.n_chunks;
+    a.image = static_cast<const uint8_t *>(window_base) - w.src_lo;  // so that image + src_off lands in the window
+    a.block_digests = d_block_digests;
+    a.tensor_digests = d_tensor_digests;
+    a.n_tensors = (uint32_t)m->entries.size();
+    a.work_counters = m->d_counter;
+    a.status = m->d_status;
+    a.hints = 0;
+    a.n_counters = 1;
+    a.group = 1;
+    a.capture = 0;
+    a.keep_accum = first ? 0u : 1u;
+    cudaError_t e = launch_restore(a, s);
+    return e == cudaSuccess ? GMS_OK : cuda_fail(e);
+}
+
 }  // namespace gms
 
 extern "C" {
@@ -226,6 +294,7 @@ int gms_manifest_destroy(gms_manifest *m)
     int rc = GMS_OK;
     if (m->d_expected && cudaFree(m->d_expected) != cudaSuccess) rc = GMS_ERR_CUDA;
     if (m->d_tables && cudaFree(m->d_tables) != cudaSuccess) rc = GMS_ERR_CUDA;
+    if (m->d_by_src && cudaFree(m->d_by_src) != cudaSuccess) rc = GMS_ERR_CUDA;
     delete m;
     return rc;
 }
@@ -297,6 +366,7 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
     a.n_counters = 1;
     a.group = 1;
     a.capture = capture ? 1u : 0u;
+    a.keep_accum = 0;
     GMS_CUDA(store ? gms::launch_restore(a, static_cast<cudaStream_t>(stream))
                    : gms::launch_digest(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
@@ -489,6 +559,7 @@ const char *gms_strerror(int status)
     case GMS_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case GMS_ERR_STATE: return "manifest lacks device tables or recorded digests";
     case GMS_ERR_ARG: return "argument out of range";
+    case GMS_ERR_IO: return "a file read failed or the file is shorter than the image";
     case GMS_ERR_TOO_LARGE: return "size exceeds the fixed capacity of the no-allocation entry point (GMS_NOALLOC_MAX_BLOCKS)";
     default: return "unknown status";
     }

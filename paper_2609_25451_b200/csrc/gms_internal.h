@@ -5,6 +5,8 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstdlib>
+#include <vector>
+
 #include <cuda_runtime.h>
 
 namespace gms {
@@ -53,6 +55,7 @@ struct StreamArgs {
     uint32_t n_counters;           // filled in by the launcher
     uint32_t group;                // filled in by the launcher
     uint32_t capture;              // 1: gather allocations into the image (restore kernel with roles swapped)
+    uint32_t keep_accum;           // 1: a later window of a windowed restore (accumulators and status are kept)
 };
 
 struct KvArgs {
@@ -91,7 +94,25 @@ constexpr uint32_t kVerifySegBlocks = 2048;  // digest slots compared by one CTA
 cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s);
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s);
 
+// A window of a restore that is fed piecewise (file -> pinned buffer -> device): a run of the
+// chunk list sorted by source offset whose sources all lie in image bytes [src_lo, src_hi).
+struct SrcWindow {
+    uint32_t first_chunk, n_chunks;
+    uint64_t src_lo, src_hi;
+};
+
 void count_launches(uint32_t n);  // bumps the process-wide launch counter
 int report_cuda_error(cudaError_t e);  // records the text for gms_last_cuda_error(); returns GMS_ERR_CUDA
 
+}  // namespace gms
+
+struct gms_manifest;
+namespace gms {
+// Cuts the manifest's work into windows of at most `buffer_bytes` of image each (building, once,
+// a device copy of the chunk list sorted by source offset).  Returns a GMS_* status.
+int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vector<SrcWindow> *out);
+// Enqueues the restore of one window; `window_base` is the device-accessible address of image byte w.src_lo.
+int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void *window_base, bool first,
+                           uint64_t *d_block_digests, uint64_t *d_tensor_digests, cudaStream_t s);
+uint64_t manifest_n_tensors(const gms_manifest *m);
 }  // namespace gms

@@ -1,0 +1,264 @@
+// gms_restore_fd: storage -> pinned host buffers -> device allocations, pipelined.
+//
+// Section 4 (GMS paragraph) has a read-write client repopulate a cold service "from storage in
+// parallel with process restoration"; Section 3.1 prices that at S / B_eff and Section 3.3 notes that
+// runtime-state restoration leaves storage bandwidth unused.  This file is that leg: the snapshot
+// image is never resident as a whole.  A small ring of pinned, device-mapped buffers is filled by a
+// pool of reader threads (pread), and as soon as a buffer holds a window of the image the restore
+// kernel is launched on the chunks whose sources lie in that window, reading the pinned buffer
+// across the host link and scattering + digesting as usual.  Reading window k+1 overlaps the kernel
+// of window k; a buffer is refilled only after the kernel that read it has finished (CUDA event).
+// All waiting is on the host (condition variables, cudaEventSynchronize); no kernel waits for a flag.
+#include <condition_variable>
+#include <cerrno>
+#include <chrono>
+#include <deque>
+#include <functional>
+#include <mutex>
+#include <thread>
+#include <vector>
+
+#include <unistd.h>
+
+#include "../../include/gms.h"
+#include "gms_internal.h"
+
+namespace {
+
+class ReaderPool {
+  public:
+    explicit ReaderPool(uint32_t n)
+    {
+        for (uint32_t i = 0; i < n; ++i) threads_.emplace_back([this] { run(); });
+    }
+    ~ReaderPool()
+    {
+        {
+            std::lock_guard<std::mutex> l(mu_);
+            stop_ = true;
+        }
+        cv_.notify_all();
+        for (auto &t : threads_) t.join();
+    }
+    void submit(std::function<void()> f)
+    {
+        {
+            std::lock_guard<std::mutex> l(mu_);
+            q_.push_back(std::move(f));
+        }
+        cv_.notify_one();
+    }
+    uint32_t size() const { return (uint32_t)threads_.size(); }
+
+  private:
+    void run()
+    {
+        for (;;) {
+            std::function<void()> f;
+            {
+                std::unique_lock<std::mutex> l(mu_);
+                cv_.wait(l, [this] { return stop_ || !q_.empty(); });
+                if (q_.empty()) return;
+                f = std::move(q_.front());
+                q_.pop_front();
+            }
+            f();
+        }
+    }
+    std::mutex mu_;
+    std::condition_variable cv_;
+    std::deque<std::function<void()>> q_;
+    std::vector<std::thread> threads_;
+    bool stop_ = false;
+};
+
+// completion state of the reads of one window
+struct WindowReads {
+    std::mutex mu;
+    std::condition_variable cv;
+    uint32_t pending = 0;
+    int error = 0;  // errno of a failed read, or -1 for an unexpected end of file
+};
+
+double now_s()
+{
+    return std::chrono::duration<double>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+
+}  // namespace
+
+struct gms_pipe {
+    uint32_t n_buffers = 0;
+    uint64_t buffer_bytes = 0;
+    std::vector<void *> host;    // pinned buffers
+    std::vector<void *> dview;   // their device-side addresses
+    std::vector<cudaEvent_t> done;
+    ReaderPool *pool = nullptr;
+    std::mutex busy;             // one restore at a time per pipe
+};
+
+extern "C" {
+
+int gms_pipe_create(uint32_t n_buffers, uint64_t buffer_bytes, uint32_t n_readers, gms_pipe **out)
+{
+    if (!out) return GMS_ERR_NULL;
+    *out = nullptr;
+    if (n_buffers < 2 || n_buffers > 64 || n_readers < 1 || n_readers > 256) return GMS_ERR_ARG;
+    if (buffer_bytes < (1ull << 20) || (buffer_bytes & 4095u)) return GMS_ERR_ARG;
+    gms_pipe *p = new (std::nothrow) gms_pipe();
+    if (!p) return GMS_ERR_NOMEM;
+    p->n_buffers = n_buffers;
+    p->buffer_bytes = buffer_bytes;
+    int rc = GMS_OK;
+    for (uint32_t b = 0; b < n_buffers && rc == GMS_OK; ++b) {
+        void *h = nullptr, *d = nullptr;
+        cudaEvent_t ev = nullptr;
+        cudaError_t e = cudaHostAlloc(&h, buffer_bytes, cudaHostAllocMapped | cudaHostAllocPortable);
+        if (e == cudaSuccess) e = cudaHostGetDevicePointer(&d, h, 0);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            if (h) cudaFreeHost(h);
+            rc = e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : gms::report_cuda_error(e);
+            (void)cudaGetLastError();
+            break;
+        }
+        p->host.push_back(h);
+        p->dview.push_back(d);
+        p->done.push_back(ev);
+    }
+    if (rc == GMS_OK) {
+        p->pool = new (std::nothrow) ReaderPool(n_readers);
+        if (!p->pool) rc = GMS_ERR_NOMEM;
+    }
+    if (rc != GMS_OK) {
+        for (void *h : p->host) cudaFreeHost(h);
+        for (cudaEvent_t ev : p->done) cudaEventDestroy(ev);
+        delete p->pool;
+        delete p;
+        return rc;
+    }
+    *out = p;
+    return GMS_OK;
+}
+
+int gms_pipe_destroy(gms_pipe *p)
+{
+    if (!p) return GMS_OK;
+    delete p->pool;  // joins the readers
+    int rc = GMS_OK;
+    for (cudaEvent_t ev : p->done)
+        if (cudaEventDestroy(ev) != cudaSuccess) rc = GMS_ERR_CUDA;
+    for (void *h : p->host)
+        if (cudaFreeHost(h) != cudaSuccess) rc = GMS_ERR_CUDA;
+    delete p;
+    return rc;
+}
+
+int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_offset, uint64_t *d_block_digests,
+                   uint64_t *d_tensor_digests, void *stream, gms_pipe_stats *stats)
+{
+    if (!m || !p) return GMS_ERR_NULL;
+    if (fd < 0) return GMS_ERR_ARG;
+    std::lock_guard<std::mutex> one(p->busy);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<gms::SrcWindow> windows;
+    int rc = gms::manifest_src_windows(m, p->buffer_bytes, &windows);
+    if (rc != GMS_OK) return rc;
+    const double t_start = now_s();
+    gms_pipe_stats st = {};
+    st.windows = windows.size();
+
+    if (windows.empty()) {  // nothing to move: still clear the accumulators
+        gms::SrcWindow none = {0, 0, 0, 0};
+        rc = gms::manifest_launch_window(m, none, p->dview[0], true, d_block_digests, d_tensor_digests, s);
+    }
+
+    std::vector<WindowReads> reads(windows.size());
+    const uint32_t n_readers = p->pool->size();
+    size_t next_read = 0, next_launch = 0;
+    int io_error = 0;
+    while (rc == GMS_OK && next_launch < windows.size()) {
+        // start reads as far ahead as the ring allows
+        while (next_read < windows.size() && next_read < next_launch + p->n_buffers) {
+            const uint32_t b = (uint32_t)(next_read % p->n_buffers);
+            if (next_read >= p->n_buffers) {  // the kernel that read this buffer last must be done with it
+                const double t0 = now_s();
+                cudaError_t e = cudaEventSynchronize(p->done[b]);
+                st.wait_gpu_seconds += now_s() - t0;
+                if (e != cudaSuccess) {
+                    rc = gms::report_cuda_error(e);
+                    break;
+                }
+            }
+            const gms::SrcWindow &w = windows[next_read];
+            WindowReads &wr = reads[next_read];
+            const uint64_t len = w.src_hi - w.src_lo;
+            // slices are multiples of 1 MiB so that readers do not share pages
+            uint64_t slice = (len + n_readers - 1) / n_readers;
+            slice = (slice + (1u << 20) - 1) & ~((uint64_t)(1u << 20) - 1);
+            const uint32_t n_slices = (uint32_t)((len + slice - 1) / slice);
+            wr.pending = n_slices;
+            uint8_t *base = static_cast<uint8_t *>(p->host[b]);
+            for (uint32_t k = 0; k < n_slices; ++k) {
+                const uint64_t lo = (uint64_t)k * slice, n = std::min<uint64_t>(slice, len - lo);
+                const uint64_t foff = file_offset + w.src_lo + lo;
+                p->pool->submit([fd, base, lo, n, foff, &wr] {
+                    uint64_t got = 0;
+                    int err = 0;
+                    while (got < n) {
+                        const ssize_t r = pread(fd, base + lo + got, n - got, (off_t)(foff + got));
+                        if (r < 0) {
+                            if (errno == EINTR) continue;
+                            err = errno ? errno : -1;
+                            break;
+                        }
+                        if (r == 0) {
+                            err = -1;  // file shorter than the image
+                            break;
+                        }
+                        got += (uint64_t)r;
+                    }
+                    std::lock_guard<std::mutex> l(wr.mu);
+                    if (err && !wr.error) wr.error = err;
+                    if (--wr.pending == 0) wr.cv.notify_all();
+                });
+            }
+            st.bytes_read += len;
+            ++next_read;
+        }
+        if (rc != GMS_OK) break;
+        // wait for the window to be launched next, then launch it
+        {
+            WindowReads &wr = reads[next_launch];
+            const double t0 = now_s();
+            std::unique_lock<std::mutex> l(wr.mu);
+            wr.cv.wait(l, [&wr] { return wr.pending == 0; });
+            st.wait_read_seconds += now_s() - t0;
+            if (wr.error) {
+                io_error = wr.error;
+                break;
+            }
+        }
+        const uint32_t b = (uint32_t)(next_launch % p->n_buffers);
+        rc = gms::manifest_launch_window(m, windows[next_launch], p->dview[b], next_launch == 0, d_block_digests,
+                                         d_tensor_digests, s);
+        if (rc == GMS_OK) {
+            cudaError_t e = cudaEventRecord(p->done[b], s);
+            if (e != cudaSuccess) rc = gms::report_cuda_error(e);
+        }
+        ++next_launch;
+    }
+    // drain: reads still in flight must not outlive this call (they write into the pipe's buffers and use `reads`)
+    for (size_t w = 0; w < next_read; ++w) {
+        std::unique_lock<std::mutex> l(reads[w].mu);
+        reads[w].cv.wait(l, [&] { return reads[w].pending == 0; });
+    }
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess && rc == GMS_OK) rc = gms::report_cuda_error(e);
+    st.total_seconds = now_s() - t_start;
+    if (stats) *stats = st;
+    if (io_error) return GMS_ERR_IO;
+    return rc;
+}
+
+}  // extern "C"

@@ -578,7 +578,10 @@ cudaError_t launch_stream(const StreamArgs &a, cudaStream_t s)
     Geometry g;
     cudaError_t e = get_geometry(kStore ? kRestore : kDigest, &g);
     if (e) return e;
-    if ((e = prologue(a.tensor_digests, a.n_tensors, a.work_counters, g.counters, a.status, 1, s))) return e;
+    // a windowed restore keeps the tensor-digest accumulators and the status word of its earlier windows
+    if ((e = prologue(a.keep_accum ? nullptr : a.tensor_digests, a.n_tensors, a.work_counters, g.counters, a.status,
+                      a.keep_accum ? 0 : 1, s)))
+        return e;
     if (a.n_chunks == 0) return cudaSuccess;
     StreamArgs b = a;
     b.hints = g.hints;

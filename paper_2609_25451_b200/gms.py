@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libgms.so")
 BLOCK_BYTES = 4096
 OK = 0
 ERR_NULL, ERR_ALIGN, ERR_RANGE, ERR_OVERLAP, ERR_DUP_ID, ERR_NOMEM = -1, -2, -3, -4, -5, -6
-ERR_CUDA, ERR_KIND, ERR_TIMEOUT, ERR_STATE, ERR_ARG, ERR_TOO_LARGE = -7, -8, -9, -10, -11, -12
+ERR_CUDA, ERR_KIND, ERR_TIMEOUT, ERR_STATE, ERR_ARG, ERR_TOO_LARGE, ERR_IO = -7, -8, -9, -10, -11, -12, -13
 NOALLOC_MAX_BLOCKS = 4194304
 SRC_DEVICE, SRC_HOST_MAPPED = 0, 1
 BUILD_HOST_ONLY = 1
@@ -32,6 +32,7 @@ EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
     "gms_verify", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_host_image_alloc", "gms_host_image_free",
+    "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd",
     "gms_launch_geometry", "gms_kernel_launches", "gms_set_device", "gms_strerror", "gms_last_cuda_error", "gms_version",
 )
 
@@ -81,6 +82,9 @@ def lib():
             "gms_kv_capture": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
             "gms_host_image_alloc": (i, [u64, pp, pp]),
             "gms_host_image_free": (i, [p]),
+            "gms_pipe_create": (i, [u32, u64, u32, pp]),
+            "gms_pipe_destroy": (i, [p]),
+            "gms_restore_fd": (i, [p, p, i, u64, p, p, p, p]),
             "gms_launch_geometry": (i, [pu32, pu32, pu32]),
             "gms_kernel_launches": (u64, []),
             "gms_set_device": (i, [i]),
@@ -228,6 +232,39 @@ def gms_host_image_alloc(nbytes: int):
 
 def gms_host_image_free(host_ptr: int):
     _check(lib().gms_host_image_free(host_ptr), "gms_host_image_free")
+
+
+class PipeStats(C.Structure):
+    _fields_ = [("windows", C.c_uint64), ("bytes_read", C.c_uint64), ("wait_read_seconds", C.c_double),
+                ("wait_gpu_seconds", C.c_double), ("total_seconds", C.c_double)]
+
+
+class Pipe:
+    """Owner of a ``gms_pipe*`` (ring of pinned buffers + reader threads)."""
+
+    def __init__(self, handle):
+        self.handle = handle
+
+    def close(self):
+        if self.handle:
+            lib().gms_pipe_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+
+def gms_pipe_create(n_buffers: int, buffer_bytes: int, n_readers: int) -> Pipe:
+    out = C.c_void_p()
+    _check(lib().gms_pipe_create(n_buffers, int(buffer_bytes), n_readers, C.byref(out)), "gms_pipe_create")
+    return Pipe(out.value)
+
+
+def gms_restore_fd(m: Manifest, pipe: Pipe, fd: int, file_offset: int, d_block_digests, d_tensor_digests, stream=None) -> dict:
+    """Synchronous; returns the call's statistics as a dict."""
+    st = PipeStats()
+    _check(lib().gms_restore_fd(m.handle, pipe.handle, int(fd), int(file_offset), _dev(d_block_digests),
+                                _dev(d_tensor_digests), _stream(stream), C.byref(st)), "gms_restore_fd")
+    return {k: getattr(st, k) for k, _ in PipeStats._fields_}
 
 
 def gms_launch_geometry():

@@ -1,0 +1,113 @@
+"""gms_restore_fd: restore fed from a file through a ring of pinned buffers.  The result must be
+exactly what gms_restore produces from the same bytes, so the oracle's restore of the file's
+contents is the reference: destination bytes, block digests, tensor digests, bit-exact -- with
+buffers far smaller than the tensors (tensors span many windows), a non-zero file offset, odd
+sizes, and the error paths (short file, bad arguments)."""
+import ctypes
+import os
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from paper_2609_25451_b200 import gms  # noqa: E402
+from paper_2609_25451_b200 import workloads as W  # noqa: E402
+
+from gpu_harness import FILL, DeviceWorkload, oracle_record  # noqa: E402
+
+
+def test_pipe_argument_checks_need_no_gpu():
+    out = ctypes.c_void_p()
+    L = gms.lib()
+    assert L.gms_pipe_create(1, 1 << 20, 4, ctypes.byref(out)) == gms.ERR_ARG      # fewer than 2 buffers
+    assert L.gms_pipe_create(2, 4096, 4, ctypes.byref(out)) == gms.ERR_ARG          # buffer below 1 MiB
+    assert L.gms_pipe_create(2, (1 << 20) + 8, 4, ctypes.byref(out)) == gms.ERR_ARG  # not a multiple of 4096
+    assert L.gms_pipe_create(2, 1 << 20, 0, ctypes.byref(out)) == gms.ERR_ARG       # no readers
+    assert L.gms_pipe_create(2, 1 << 20, 4, None) == gms.ERR_NULL
+    assert L.gms_pipe_destroy(None) == gms.OK
+    assert L.gms_restore_fd(None, None, 0, 0, None, None, None, None) == gms.ERR_NULL
+    assert "file" in gms.gms_strerror(gms.ERR_IO)
+
+
+def _write_image(path, image: np.ndarray, file_offset: int):
+    with open(path, "wb") as f:
+        f.write(b"\xAB" * file_offset)
+        f.write(image.tobytes())
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("n_buffers,buffer_mib,n_readers,file_offset", [(2, 1, 1, 0), (3, 2, 4, 4096 + 16), (4, 16, 8, 512)])
+def test_restore_fd_equals_restore_of_the_same_bytes(oracle, tmp_path, n_buffers, buffer_mib, n_readers, file_offset):
+    w = W.mixed_manifest(n_small=1500, n_large=3, large_bytes=(7 << 20) + 40, round16=False, seed=123)
+    image = W.random_bytes_host(w.image_bytes, seed=77)
+    slab_h = np.full(w.slab_bytes, FILL, np.uint8)
+    rc, obd, otd = oracle.restore(oracle_record(oracle, w), image, slab_h)
+    assert rc == 0
+    path = str(tmp_path / "image.bin")
+    _write_image(path, image, file_offset)
+    d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    pipe = gms.gms_pipe_create(n_buffers, buffer_mib << 20, n_readers)
+    fd = os.open(path, os.O_RDONLY)
+    try:
+        for _ in range(2):  # twice: the second call must not be disturbed by what the first left in the buffers
+            d.slab.fill_(FILL)
+            d.reset_outputs()
+            st = gms.gms_restore_fd(d.m, pipe, fd, file_offset, d.bd_ptr(), d.td_ptr())
+            assert gms.gms_last_device_status(d.m) == 0
+            from gpu_harness import payload_of
+
+            assert np.array_equal(d.slab_host(), slab_h), "destination bytes (or guard bands) differ"
+            assert np.array_equal(payload_of(d.bd, d.nb), obd) and np.array_equal(payload_of(d.td, d.nt), otd)
+            assert st["windows"] >= w.image_bytes // (buffer_mib << 20) and st["bytes_read"] <= w.image_bytes
+    finally:
+        os.close(fd)
+        pipe.close()
+        d.close()
+
+
+@pytest.mark.gpu
+def test_restore_fd_reports_a_short_file(tmp_path):
+    w = W.pack_layout("short", [3 << 20, 5 << 20, 100], seed=5)
+    image = W.random_bytes_host(w.image_bytes, seed=1)
+    path = str(tmp_path / "short.bin")
+    _write_image(path, image[: w.image_bytes - (2 << 20)], 0)  # the file ends 2 MiB early
+    d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    pipe = gms.gms_pipe_create(2, 1 << 20, 2)
+    fd = os.open(path, os.O_RDONLY)
+    try:
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_restore_fd(d.m, pipe, fd, 0, None, None)
+        assert ei.value.status == gms.ERR_IO
+        # the pipe and the manifest remain usable after the error
+        os.close(fd)
+        _write_image(path, image, 0)
+        fd = os.open(path, os.O_RDONLY)
+        gms.gms_restore_fd(d.m, pipe, fd, 0, None, None)
+        for r in w.rows:
+            s, o, n = int(r["src_offset"]), int(r["dst_offset"]), int(r["nbytes"])
+            assert np.array_equal(d.slab[o:o + n].cpu().numpy(), image[s:s + n])
+    finally:
+        os.close(fd)
+        pipe.close()
+        d.close()
+
+
+@pytest.mark.gpu
+def test_restore_fd_empty_manifest(tmp_path):
+    w = W.pack_layout("empty", [0, 0], seed=1)
+    path = str(tmp_path / "e.bin")
+    _write_image(path, np.zeros(16, np.uint8), 0)
+    d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    pipe = gms.gms_pipe_create(2, 1 << 20, 1)
+    fd = os.open(path, os.O_RDONLY)
+    try:
+        d.reset_outputs()
+        st = gms.gms_restore_fd(d.m, pipe, fd, 0, d.bd_ptr(), d.td_ptr())
+        from gpu_harness import payload_of
+
+        assert st["windows"] == 0 and (payload_of(d.td, d.nt) == 0).all()
+    finally:
+        os.close(fd)
+        pipe.close()
+        d.close()
