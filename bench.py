@@ -1,13 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the GMS restore / digest / verify path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 8b|mixed|tiny|kv|host70b]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 8b|mixed|tiny|kv|host70b|capture|file]
     python bench.py --impl reference ...      # the CPU oracle on this host's cores
 
 One *step* is one pass of the whole hot path over one synthetic snapshot:
     gms_digest  (digest the preserved allocations in place)   -> gms_verify
     gms_restore (scatter the device-staged image, fused digest) -> gms_verify
-(`kv`: one gms_kv_restore; `host70b`: one host-sourced gms_restore + gms_verify).
+(`kv`: one gms_kv_restore; `host70b`: one host-sourced gms_restore + gms_verify; `capture`: gms_capture +
+gms_verify; `file`: gms_restore_fd from a file through pinned buffers).
 The default workload is the Llama-3-8B-shaped weight manifest (291 tensors, 16.06 GB of random
 bf16 bit patterns); image and destinations are resident in HBM when the timed region starts and are
 ~250x larger than L2, so no L2 flush is needed between iterations.
@@ -40,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 DATASHEET_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the restore kernel, per payload byte, from the
 # ncu capture summarised under profiles/ (None until captured); scaled by the payload of a launch.
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"restore": 1.984, "digest": 1.006, "kv_restore": None}
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"restore": 1.983, "digest": 1.008, "kv_restore": 1.919, "capture": 1.983}
 
 
 def parse_args():
@@ -59,6 +60,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target CPU time of the oracle sample")
     ap.add_argument("--host-gib", type=float, default=32.0, help="host70b: size of the pinned host image")
+    ap.add_argument("--kv-gb", type=float, default=60.0, help="kv: size of the paged pool (a small pool is used for ncu captures)")
     return ap.parse_args()
 
 
@@ -487,7 +489,7 @@ def main():
 
     sampler = ClockSampler(local_rank)
     if args.workload == "kv":
-        bench = KvBench(torch, gms, W, dev)
+        bench = KvBench(torch, gms, W, dev, pool_bytes=args.kv_gb * 1e9)
     elif args.workload in ("host70b", "file"):
         bench = None
     elif args.workload == "capture":

@@ -6,10 +6,16 @@
 // no tensor cores; what matters is bytes in flight, full-line transactions and
 // no per-tensor launches.
 //
-// Design.  One CTA per SM, a dozen warps per CTA, and every warp is its own
-// small pipeline with no CTA-wide synchronisation at all:
-//   * the warp claims a chunk (<= 32 digest blocks of one tensor) from the
-//     manifest's work list with one atomicAdd -- no warp ever waits for another;
+// Design.  One CTA per SM (8 warps x 6 ring slots for the copying kernels, 16 x 3
+// for digest-only), and every warp is its own small pipeline with no CTA-wide
+// synchronisation at all:
+//   * the warp claims a chunk (by default 4 digest blocks = 16 KiB of one tensor,
+//     at most 32) from the manifest's work list with one atomicAdd, drawn one
+//     chunk ahead of its use so the atomic's latency is never exposed -- no warp
+//     ever waits for another.  The copying kernels draw from a single counter:
+//     chunks are then started in strict list (= address) order, all bytes in
+//     flight lie in a narrow moving window of the image, and HBM rewards that
+//     (measured: +3..5 % over round-robin or interleaved counters);
 //   * lane 0 moves each 4 KiB digest block with a 1-D bulk async copy (TMA)
 //     global -> shared, completion signalled on an mbarrier, up to S-1 blocks
 //     ahead of the block being digested (S ring slots per warp);
@@ -131,6 +137,7 @@ __device__ __forceinline__ uint64_t mix_full(uint64_t z)
 // mix(w ^ c) without its last xor-shift; cfold = c ^ (c >> 30).
 __device__ __forceinline__ uint64_t mix_head(uint64_t w, uint64_t cfold)
 {
+    // (spelling the products on 32-bit halves with mul.hi executes 5 % fewer instructions but runs 7 % slower)
     uint64_t z = (w ^ (w >> 30) ^ cfold) * kM1;
     z = (z ^ (z >> 27)) * kM2;
     return z;
