@@ -304,6 +304,53 @@ int gms_pipe_destroy(gms_pipe *p);
 int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_offset, uint64_t *d_block_digests,
                    uint64_t *d_tensor_digests, void *stream, gms_pipe_stats *stats);
 
+/*
+ * gms_service_* -- the substrate under the destinations: Section 4, GMS paragraph (physical
+ * allocations made with cuMemCreate, a first-fit suballocator over 2 GiB slabs with dedicated
+ * slabs for larger allocations, permissions set per slab) and Section 3.2 (ownership protocol:
+ * EMPTY -> RW, one writer populates -> COMMITTED, immutable -> RO while n >= 1 readers hold it;
+ * a writer that gives up before commit discards everything; write access returns after the last
+ * reader has left; read-only is enforced with cuMemSetAccess).  One process, current device; the
+ * separate service process and descriptor passing of the paper are not part of this library.
+ *   create      slab_bytes = 0 means 2 GiB; GMS_SERVICE_DRY_RUN keeps the books without any CUDA
+ *               call (addresses are made up and must not be dereferenced)
+ *   acquire_rw  EMPTY -> RW, or COMMITTED -> RW (contents and addresses kept, slabs writable again);
+ *               GMS_ERR_STATE while a writer or readers hold the service
+ *   alloc       RW only; 256-byte aligned device address, first fit over the slabs, a dedicated slab
+ *               if nbytes exceeds the slab size; individual allocations are never freed, only all
+ *               at once (abort / destroy)
+ *   commit      RW -> COMMITTED: the device is synchronised, then every slab becomes read-only
+ *   abort       RW -> EMPTY: every slab is unmapped and released
+ *   acquire_ro / release_ro   COMMITTED <-> RO with a reader count
+ * After commit the addresses may be read by anything (gms_digest, gms_capture, an engine's
+ * kernels); writing to them faults the writing context, so gms_restore / gms_kv_restore must only
+ * target them in state RW (gms_service_access tells which it is).  Errors: NULL, ARG, STATE, NOMEM,
+ * RANGE (access: not an address of this service), CUDA.
+ */
+#define GMS_STATE_EMPTY 0u
+#define GMS_STATE_RW 1u
+#define GMS_STATE_COMMITTED 2u
+#define GMS_STATE_RO 3u
+#define GMS_SERVICE_DRY_RUN 1u
+typedef struct gms_service gms_service; /* opaque */
+typedef struct {
+    uint32_t state, readers;
+    uint64_t n_slabs, n_dedicated; /* slabs in all, and those holding one oversized allocation */
+    uint64_t slab_bytes;           /* regular slab size after rounding to the mapping granularity */
+    uint64_t bytes_reserved;       /* sum of slab sizes                                           */
+    uint64_t bytes_allocated;      /* sum of (256-byte rounded) allocation sizes                  */
+} gms_service_stats;
+int gms_service_create(uint64_t slab_bytes, uint32_t flags, gms_service **out);
+int gms_service_destroy(gms_service *s);
+int gms_service_acquire_rw(gms_service *s);
+int gms_service_alloc(gms_service *s, uint64_t nbytes, void **dptr);
+int gms_service_commit(gms_service *s);
+int gms_service_abort(gms_service *s);
+int gms_service_acquire_ro(gms_service *s);
+int gms_service_release_ro(gms_service *s);
+int gms_service_info(gms_service *s, gms_service_stats *out);
+int gms_service_access(gms_service *s, const void *dptr, uint32_t *writable);
+
 /* Launch geometry of the streaming kernels on the current device (for reporting). */
 int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *smem_bytes);
 /* Number of kernels this library has launched in this process so far (for reporting). */

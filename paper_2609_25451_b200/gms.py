@@ -33,6 +33,8 @@ EXPORTS = (
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
     "gms_verify", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_host_image_alloc", "gms_host_image_free",
     "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd",
+    "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
+    "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
     "gms_launch_geometry", "gms_kernel_launches", "gms_set_device", "gms_strerror", "gms_last_cuda_error", "gms_version",
 )
 
@@ -85,6 +87,16 @@ def lib():
             "gms_pipe_create": (i, [u32, u64, u32, pp]),
             "gms_pipe_destroy": (i, [p]),
             "gms_restore_fd": (i, [p, p, i, u64, p, p, p, p]),
+            "gms_service_create": (i, [u64, u32, pp]),
+            "gms_service_destroy": (i, [p]),
+            "gms_service_acquire_rw": (i, [p]),
+            "gms_service_alloc": (i, [p, u64, pp]),
+            "gms_service_commit": (i, [p]),
+            "gms_service_abort": (i, [p]),
+            "gms_service_acquire_ro": (i, [p]),
+            "gms_service_release_ro": (i, [p]),
+            "gms_service_info": (i, [p, p]),
+            "gms_service_access": (i, [p, p, pu32]),
             "gms_launch_geometry": (i, [pu32, pu32, pu32]),
             "gms_kernel_launches": (u64, []),
             "gms_set_device": (i, [i]),
@@ -265,6 +277,74 @@ def gms_restore_fd(m: Manifest, pipe: Pipe, fd: int, file_offset: int, d_block_d
     _check(lib().gms_restore_fd(m.handle, pipe.handle, int(fd), int(file_offset), _dev(d_block_digests),
                                 _dev(d_tensor_digests), _stream(stream), C.byref(st)), "gms_restore_fd")
     return {k: getattr(st, k) for k, _ in PipeStats._fields_}
+
+
+STATE_EMPTY, STATE_RW, STATE_COMMITTED, STATE_RO = 0, 1, 2, 3
+SERVICE_DRY_RUN = 1
+
+
+class ServiceStats(C.Structure):
+    _fields_ = [("state", C.c_uint32), ("readers", C.c_uint32), ("n_slabs", C.c_uint64), ("n_dedicated", C.c_uint64),
+                ("slab_bytes", C.c_uint64), ("bytes_reserved", C.c_uint64), ("bytes_allocated", C.c_uint64)]
+
+
+class Service:
+    """Owner of a ``gms_service*``."""
+
+    def __init__(self, handle):
+        self.handle = handle
+
+    def close(self):
+        if self.handle:
+            lib().gms_service_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+
+def gms_service_create(slab_bytes: int = 0, flags: int = 0) -> Service:
+    out = C.c_void_p()
+    _check(lib().gms_service_create(int(slab_bytes), flags, C.byref(out)), "gms_service_create")
+    return Service(out.value)
+
+
+def gms_service_acquire_rw(s: Service):
+    _check(lib().gms_service_acquire_rw(s.handle), "gms_service_acquire_rw")
+
+
+def gms_service_alloc(s: Service, nbytes: int) -> int:
+    p = C.c_void_p()
+    _check(lib().gms_service_alloc(s.handle, int(nbytes), C.byref(p)), "gms_service_alloc")
+    return p.value
+
+
+def gms_service_commit(s: Service):
+    _check(lib().gms_service_commit(s.handle), "gms_service_commit")
+
+
+def gms_service_abort(s: Service):
+    _check(lib().gms_service_abort(s.handle), "gms_service_abort")
+
+
+def gms_service_acquire_ro(s: Service):
+    _check(lib().gms_service_acquire_ro(s.handle), "gms_service_acquire_ro")
+
+
+def gms_service_release_ro(s: Service):
+    _check(lib().gms_service_release_ro(s.handle), "gms_service_release_ro")
+
+
+def gms_service_info(s: Service) -> dict:
+    st = ServiceStats()
+    _check(lib().gms_service_info(s.handle, C.byref(st)), "gms_service_info")
+    return {k: getattr(st, k) for k, _ in ServiceStats._fields_}
+
+
+def gms_service_access(s: Service, dptr: int) -> bool:
+    """True if the address is currently mapped writable."""
+    w = C.c_uint32()
+    _check(lib().gms_service_access(s.handle, int(dptr), C.byref(w)), "gms_service_access")
+    return bool(w.value)
 
 
 def gms_launch_geometry():

@@ -1,0 +1,180 @@
+"""gms_service_*: service-owned slabs with the paper's ownership protocol (EMPTY -> RW -> COMMITTED
+<-> RO), a first-fit suballocator over fixed-size slabs and dedicated slabs for oversized requests.
+
+CPU part (dry-run backend, no CUDA call): the state machine accepts exactly the transitions of the
+protocol, and the allocator's addresses are aligned, disjoint, first-fit and inside their slabs.
+GPU part: destinations carved from real VMM slabs take a restore (parity with the oracle), become
+read-only at commit (checked through cuMemGetAccess, never by attempting a write), can still be
+digested / verified / captured in place while readers hold them, and are writable again after the
+last reader has left.  No test writes to a read-only mapping."""
+import numpy as np
+import pytest
+
+from paper_2609_25451_b200 import gms
+from paper_2609_25451_b200 import workloads as W
+
+MiB = 1 << 20
+
+
+def status_of(fn, *a):
+    try:
+        fn(*a)
+        return gms.OK
+    except gms.GmsError as e:
+        return e.status
+
+
+def test_ownership_state_machine_dry_run():
+    s = gms.gms_service_create(8 * MiB, gms.SERVICE_DRY_RUN)
+    info = lambda: gms.gms_service_info(s)
+    assert info()["state"] == gms.STATE_EMPTY
+    # nothing but a writer may start
+    assert status_of(gms.gms_service_alloc, s, 100) == gms.ERR_STATE
+    assert status_of(gms.gms_service_commit, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_acquire_ro, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_release_ro, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_abort, s) == gms.ERR_STATE
+    gms.gms_service_acquire_rw(s)
+    assert info()["state"] == gms.STATE_RW
+    assert status_of(gms.gms_service_acquire_rw, s) == gms.ERR_STATE  # one writer only
+    assert status_of(gms.gms_service_acquire_ro, s) == gms.ERR_STATE  # no readers before commit
+    p = gms.gms_service_alloc(s, 1000)
+    assert gms.gms_service_access(s, p) is True
+    # a writer that gives up discards everything
+    gms.gms_service_abort(s)
+    assert info()["state"] == gms.STATE_EMPTY and info()["n_slabs"] == 0 and info()["bytes_allocated"] == 0
+    assert status_of(gms.gms_service_access, s, p) == gms.ERR_RANGE
+    # populate, commit, readers come and go
+    gms.gms_service_acquire_rw(s)
+    p = gms.gms_service_alloc(s, 1000)
+    gms.gms_service_commit(s)
+    assert info()["state"] == gms.STATE_COMMITTED and gms.gms_service_access(s, p) is False
+    assert status_of(gms.gms_service_alloc, s, 100) == gms.ERR_STATE  # immutable
+    assert status_of(gms.gms_service_abort, s) == gms.ERR_STATE
+    gms.gms_service_acquire_ro(s)
+    gms.gms_service_acquire_ro(s)
+    assert info()["state"] == gms.STATE_RO and info()["readers"] == 2
+    assert status_of(gms.gms_service_acquire_rw, s) == gms.ERR_STATE  # readers hold it
+    gms.gms_service_release_ro(s)
+    assert info()["state"] == gms.STATE_RO and info()["readers"] == 1
+    gms.gms_service_release_ro(s)
+    assert info()["state"] == gms.STATE_COMMITTED and info()["readers"] == 0
+    assert status_of(gms.gms_service_release_ro, s) == gms.ERR_STATE
+    # write access returns after the last reader; contents and addresses are kept
+    gms.gms_service_acquire_rw(s)
+    assert info()["state"] == gms.STATE_RW and info()["n_slabs"] == 1 and gms.gms_service_access(s, p) is True
+    s.close()
+    assert gms.lib().gms_service_create(0, 0x80, None) == gms.ERR_NULL
+
+
+def test_first_fit_suballocation_dry_run():
+    slab = 8 * MiB
+    s = gms.gms_service_create(slab, gms.SERVICE_DRY_RUN)
+    gms.gms_service_acquire_rw(s)
+    rng = np.random.default_rng(4)
+    sizes = [int(x) for x in rng.integers(1, 3 * MiB, size=40)] + [slab, slab + 1, 20 * MiB, 1, 255, 256, 257]
+    allocs = [(gms.gms_service_alloc(s, n), n) for n in sizes]
+    info = gms.gms_service_info(s)
+    assert info["slab_bytes"] == slab and info["n_dedicated"] == 2  # slab+1 and 20 MiB do not fit a regular slab
+    assert info["bytes_allocated"] == sum((n + 255) // 256 * 256 for n in sizes)
+    assert info["bytes_reserved"] >= info["bytes_allocated"]
+    spans = sorted((p, p + (n + 255) // 256 * 256) for p, n in allocs)
+    assert all(p % 256 == 0 for p, _ in spans)
+    assert all(a_end <= b_start for (_, a_end), (b_start, _) in zip(spans, spans[1:]))  # pairwise disjoint
+    # first fit: a small request goes into the first regular slab that still has a gap (here the very first
+    # slab, whose tail was too short for the request that opened the second one), not into a new slab
+    first_slab_base = allocs[0][0]
+    small = gms.gms_service_alloc(s, 64)
+    assert first_slab_base <= small < first_slab_base + slab
+    assert gms.gms_service_info(s)["n_slabs"] == info["n_slabs"]
+    assert status_of(gms.gms_service_alloc, s, 0) == gms.ERR_ARG
+    s.close()
+
+
+@pytest.mark.gpu
+def test_restore_into_slabs_commit_read_only_and_repair(oracle):
+    import torch
+
+    from gpu_harness import oracle_record
+
+    w = W.mixed_manifest(n_small=600, n_large=3, large_bytes=(9 * MiB) + 40, round16=False, seed=202)
+    image_h = W.random_bytes_host(w.image_bytes, seed=203)
+    svc = gms.gms_service_create(16 * MiB)  # small slabs so that the workload spans many of them
+    gms.gms_service_acquire_rw(svc)
+    ptrs = [gms.gms_service_alloc(svc, max(1, int(r["nbytes"]))) for r in w.rows]
+    info = gms.gms_service_info(svc)
+    assert info["n_slabs"] >= 3 and info["state"] == gms.STATE_RW
+    assert all(gms.gms_service_access(svc, p) for p in ptrs[:5])
+    image = torch.from_numpy(image_h).cuda()
+    ent = gms.make_entries((r["tensor_id"], r["src_offset"], p, r["nbytes"]) for r, p in zip(w.rows, ptrs))
+    m = gms.gms_manifest_build(ent, w.image_bytes)
+    bd = torch.zeros(m.n_blocks, dtype=torch.int64, device="cuda")
+    td = torch.zeros(m.n_tensors, dtype=torch.int64, device="cuda")
+    gms.gms_restore(m, image, gms.SRC_DEVICE, bd, td)
+    torch.cuda.synchronize()
+    # the oracle's view: same record with destinations packed on the host
+    rec = oracle_record(oracle, w)
+    slab_h = np.zeros(w.slab_bytes, np.uint8)
+    rc, obd, otd = oracle.restore(rec, image_h, slab_h)
+    assert rc == 0
+    assert np.array_equal(bd.cpu().numpy().view(np.uint64), obd) and np.array_equal(td.cpu().numpy().view(np.uint64), otd)
+    gms.gms_manifest_set_expected(m, bd)
+
+    # commit: every slab read-only (asked of the driver, not tried by writing)
+    gms.gms_service_commit(svc)
+    assert not any(gms.gms_service_access(svc, p) for p in ptrs)
+    gms.gms_service_acquire_ro(svc)
+    assert gms.gms_service_info(svc)["state"] == gms.STATE_RO
+    # a reader digests, verifies and captures the read-only allocations in place
+    bd2 = torch.zeros_like(bd)
+    td2 = torch.zeros_like(td)
+    gms.gms_digest(m, bd2, td2)
+    out = torch.zeros(2 * 8, dtype=torch.int64, device="cuda")
+    cnt = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    gms.gms_verify(m, bd2, out, 8, cnt)
+    back = torch.zeros(w.image_bytes, dtype=torch.uint8, device="cuda")
+    gms.gms_capture(m, back, gms.SRC_DEVICE, None, None)
+    torch.cuda.synchronize()
+    assert torch.equal(bd2, bd) and torch.equal(td2, td) and int(cnt.item()) == 0
+    for r in w.rows:
+        s0, n = int(r["src_offset"]), int(r["nbytes"])
+        assert torch.equal(back[s0:s0 + n], image[s0:s0 + n])
+    assert gms.gms_last_device_status(m) == 0
+    assert status_of(gms.gms_service_acquire_rw, svc) == gms.ERR_STATE
+    gms.gms_service_release_ro(svc)
+
+    # the last reader has left: a writer repairs in place (same addresses), with a different image
+    gms.gms_service_acquire_rw(svc)
+    assert all(gms.gms_service_access(svc, p) for p in ptrs)
+    image2_h = W.random_bytes_host(w.image_bytes, seed=204)
+    gms.gms_restore(m, torch.from_numpy(image2_h).cuda(), gms.SRC_DEVICE, bd, td)
+    torch.cuda.synchronize()
+    rc, obd2, otd2 = oracle.restore(rec, image2_h, slab_h)
+    assert np.array_equal(bd.cpu().numpy().view(np.uint64), obd2) and np.array_equal(td.cpu().numpy().view(np.uint64), otd2)
+    gms.gms_service_abort(svc)
+    assert gms.gms_service_info(svc)["n_slabs"] == 0
+    m.close()
+    svc.close()
+
+
+@pytest.mark.gpu
+def test_oversized_allocation_gets_a_dedicated_slab():
+    import torch
+
+    svc = gms.gms_service_create(4 * MiB)
+    gms.gms_service_acquire_rw(svc)
+    small = gms.gms_service_alloc(svc, 1 * MiB)
+    big = gms.gms_service_alloc(svc, 10 * MiB + 5)
+    info = gms.gms_service_info(svc)
+    assert info["n_slabs"] == 2 and info["n_dedicated"] == 1 and info["bytes_reserved"] >= 14 * MiB
+    # both are usable device memory
+    n = 10 * MiB + 5
+    image = torch.from_numpy(W.random_bytes_host(n + MiB, seed=9)).cuda()
+    m = gms.gms_manifest_build(gms.make_entries([(1, 0, big, n), (2, (n + 15) // 16 * 16, small, MiB - 16)]), n + MiB)
+    gms.gms_restore(m, image, gms.SRC_DEVICE, None, None)
+    back = torch.zeros(n + MiB, dtype=torch.uint8, device="cuda")
+    gms.gms_capture(m, back, gms.SRC_DEVICE, None, None)
+    torch.cuda.synchronize()
+    assert torch.equal(back[:n], image[:n])
+    m.close()
+    svc.close()
