@@ -51,6 +51,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["gms", "reference"], default="gms")
     ap.add_argument("--workload", choices=["8b", "mixed", "tiny", "kv", "host70b", "capture", "file"], default="8b")
+    ap.add_argument("--vmm", action="store_true", help="8b/mixed/tiny/capture/file: destinations from gms_service VMM slabs")
     ap.add_argument("--file-dir", default="/dev/shm", help="file: where the snapshot file is written")
     ap.add_argument("--pipe-buffers", type=int, default=4)
     ap.add_argument("--pipe-mib", type=int, default=256)
@@ -167,8 +168,19 @@ class ManifestBench:
         w = self.w
         self.image = torch.empty(w.image_bytes, dtype=torch.uint8, device=dev)
         W.fill_random_device(self.image, W.SEED_BASE + 0x100)
-        self.slab = torch.zeros(w.slab_bytes, dtype=torch.uint8, device=dev)
-        self.entries = self._entries(self.slab.data_ptr())
+        self.vmm = bool(os.environ.get("GMS_BENCH_VMM"))  # set by --vmm: destinations carved from gms_service slabs
+        if self.vmm:
+            import numpy as np
+
+            self.svc = gms.gms_service_create(0)  # 2 GiB slabs, dedicated slabs above that
+            gms.gms_service_acquire_rw(self.svc)
+            ptrs = [gms.gms_service_alloc(self.svc, max(1, int(n))) for n in w.rows["nbytes"]]
+            self.slab = None
+            self.entries = self._entries(0)
+            self.entries["dst"] = np.array(ptrs, dtype=np.uint64)
+        else:
+            self.slab = torch.zeros(w.slab_bytes, dtype=torch.uint8, device=dev)
+            self.entries = self._entries(self.slab.data_ptr())
         self.m = gms.gms_manifest_build(self.entries, w.image_bytes)
         self.bd = torch.zeros(max(self.m.n_blocks, 1), dtype=torch.int64, device=dev)
         self.td = torch.zeros(max(self.m.n_tensors, 1), dtype=torch.int64, device=dev)
@@ -221,6 +233,7 @@ class ManifestBench:
         return {"workload": f"{self.w.name}: {len(self.w.rows)} tensors, {self.payload} B payload, "
                             f"{self.m.n_blocks} digest blocks, {self.n_chunks} chunks",
                 "step": "gms_digest + gms_verify + gms_restore(device image) + gms_verify",
+                "destinations": "gms_service VMM slabs (2 GiB, first fit)" if self.vmm else "carved from one cudaMalloc slab",
                 "l2": "inputs larger than L2 (no flush)" if self.payload > (512 << 20) else "working set near L2 size; not flushed",
                 "payload_bytes": self.payload}
 
@@ -469,6 +482,8 @@ def main():
     if args.impl == "reference":
         reference_arm(args)
         return
+    if args.vmm:
+        os.environ["GMS_BENCH_VMM"] = "1"
     rank, local_rank, world = dist_env()
     import torch
     import torch.distributed as dist
