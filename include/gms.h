@@ -305,6 +305,25 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
                    uint64_t *d_tensor_digests, void *stream, gms_pipe_stats *stats);
 
 /*
+ * gms_stage_* / gms_restore_staged -- host-sourced restore with the copy engine on the link
+ * (Section 5.2: the existing tool "does not saturate PCIe"; Section 3.1: S / B_eff).  Kernel-issued
+ * reads of mapped host memory (gms_restore with GMS_SRC_HOST_MAPPED) top out below what the DMA
+ * engine reaches on the same link.  Here the pinned host image is moved window by window with
+ * cudaMemcpyAsync on an internal stream into a ring of `n_buffers` device buffers of `buffer_bytes`
+ * each (>= 1 MiB, multiple of 4096), and every landed window is scattered and digested by the
+ * restore kernel on the caller's stream while the next one is in flight; all ordering is done with
+ * stream events, no kernel waits for a flag.  Asynchronous like gms_restore: outputs are valid once
+ * `stream` has been synchronised; the host image must stay untouched until then.  Results are
+ * exactly those of gms_restore from the same bytes.  `host_image` (host) must be pinned memory.
+ * Errors: NULL, ARG, KIND (not pinned host memory), NOMEM, STATE, CUDA.
+ */
+typedef struct gms_stage gms_stage; /* opaque */
+int gms_stage_create(uint32_t n_buffers, uint64_t buffer_bytes, gms_stage **out);
+int gms_stage_destroy(gms_stage *st);
+int gms_restore_staged(const gms_manifest *m, gms_stage *st, const void *host_image, uint64_t *d_block_digests,
+                       uint64_t *d_tensor_digests, void *stream);
+
+/*
  * gms_service_* -- the substrate under the destinations: Section 4, GMS paragraph (physical
  * allocations made with cuMemCreate, a first-fit suballocator over 2 GiB slabs with dedicated
  * slabs for larger allocations, permissions set per slab) and Section 3.2 (ownership protocol:

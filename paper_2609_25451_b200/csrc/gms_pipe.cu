@@ -97,7 +97,106 @@ struct gms_pipe {
     std::mutex busy;             // one restore at a time per pipe
 };
 
+// Device-side staging ring for host images that are moved by the copy engine (gms_restore_staged).
+struct gms_stage {
+    uint32_t n_buffers = 0;
+    uint64_t buffer_bytes = 0;
+    std::vector<void *> dev;            // device buffers
+    std::vector<cudaEvent_t> copied;    // buffer b holds its window (recorded on the copy stream)
+    std::vector<cudaEvent_t> consumed;  // the kernel that read buffer b has finished (recorded on the caller's stream)
+    cudaStream_t copy_stream = nullptr;
+    uint64_t uses = 0;                  // windows pushed through the ring so far (across calls)
+    std::mutex busy;
+};
+
 extern "C" {
+
+int gms_stage_create(uint32_t n_buffers, uint64_t buffer_bytes, gms_stage **out)
+{
+    if (!out) return GMS_ERR_NULL;
+    *out = nullptr;
+    if (n_buffers < 2 || n_buffers > 64) return GMS_ERR_ARG;
+    if (buffer_bytes < (1ull << 20) || (buffer_bytes & 4095u)) return GMS_ERR_ARG;
+    gms_stage *st = new (std::nothrow) gms_stage();
+    if (!st) return GMS_ERR_NOMEM;
+    st->n_buffers = n_buffers;
+    st->buffer_bytes = buffer_bytes;
+    cudaError_t e = cudaStreamCreateWithFlags(&st->copy_stream, cudaStreamNonBlocking);
+    for (uint32_t b = 0; b < n_buffers && e == cudaSuccess; ++b) {
+        void *d = nullptr;
+        cudaEvent_t a = nullptr, c = nullptr;
+        e = cudaMalloc(&d, buffer_bytes);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&a, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c, cudaEventDisableTiming);
+        if (d) st->dev.push_back(d);
+        if (a) st->copied.push_back(a);
+        if (c) st->consumed.push_back(c);
+    }
+    if (e != cudaSuccess) {
+        const int rc = e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : gms::report_cuda_error(e);
+        (void)cudaGetLastError();
+        for (void *d : st->dev) cudaFree(d);
+        for (cudaEvent_t ev : st->copied) cudaEventDestroy(ev);
+        for (cudaEvent_t ev : st->consumed) cudaEventDestroy(ev);
+        if (st->copy_stream) cudaStreamDestroy(st->copy_stream);
+        delete st;
+        return rc;
+    }
+    *out = st;
+    return GMS_OK;
+}
+
+int gms_stage_destroy(gms_stage *st)
+{
+    if (!st) return GMS_OK;
+    int rc = GMS_OK;
+    if (cudaStreamSynchronize(st->copy_stream) != cudaSuccess) rc = GMS_ERR_CUDA;
+    for (cudaEvent_t ev : st->consumed)
+        if (cudaEventSynchronize(ev) != cudaSuccess) rc = GMS_ERR_CUDA;
+    for (void *d : st->dev)
+        if (cudaFree(d) != cudaSuccess) rc = GMS_ERR_CUDA;
+    for (cudaEvent_t ev : st->copied) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : st->consumed) cudaEventDestroy(ev);
+    cudaStreamDestroy(st->copy_stream);
+    delete st;
+    return rc;
+}
+
+int gms_restore_staged(const gms_manifest *m, gms_stage *st, const void *host_image, uint64_t *d_block_digests,
+                       uint64_t *d_tensor_digests, void *stream)
+{
+    if (!m || !st) return GMS_ERR_NULL;
+    std::lock_guard<std::mutex> one(st->busy);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<gms::SrcWindow> windows;
+    int rc = gms::manifest_src_windows(m, st->buffer_bytes, &windows);
+    if (rc != GMS_OK) return rc;
+    if (!windows.empty() && !host_image) return GMS_ERR_NULL;
+    if (windows.empty()) {
+        gms::SrcWindow none = {0, 0, 0, 0};
+        return gms::manifest_launch_window(m, none, st->dev[0], true, d_block_digests, d_tensor_digests, s);
+    }
+    cudaPointerAttributes at;
+    cudaError_t e = cudaPointerGetAttributes(&at, host_image);
+    if (e != cudaSuccess) return gms::report_cuda_error(e);
+    if (at.type != cudaMemoryTypeHost) return GMS_ERR_KIND;  // must be pinned host memory: the copy engine reads it
+    const uint8_t *host = static_cast<const uint8_t *>(host_image);
+    for (size_t w = 0; w < windows.size(); ++w) {
+        const uint32_t b = (uint32_t)(st->uses % st->n_buffers);
+        // copy engine: wait until the kernel that last read this buffer is done, then fill it
+        if (st->uses >= st->n_buffers && (e = cudaStreamWaitEvent(st->copy_stream, st->consumed[b], 0)) != cudaSuccess) break;
+        const uint64_t len = windows[w].src_hi - windows[w].src_lo;
+        if ((e = cudaMemcpyAsync(st->dev[b], host + windows[w].src_lo, len, cudaMemcpyHostToDevice, st->copy_stream)) != cudaSuccess) break;
+        if ((e = cudaEventRecord(st->copied[b], st->copy_stream)) != cudaSuccess) break;
+        // caller's stream: wait for the window, restore from it, release the buffer
+        if ((e = cudaStreamWaitEvent(s, st->copied[b], 0)) != cudaSuccess) break;
+        rc = gms::manifest_launch_window(m, windows[w], st->dev[b], w == 0, d_block_digests, d_tensor_digests, s);
+        if (rc != GMS_OK) return rc;
+        if ((e = cudaEventRecord(st->consumed[b], s)) != cudaSuccess) break;
+        ++st->uses;
+    }
+    return e == cudaSuccess ? GMS_OK : gms::report_cuda_error(e);
+}
 
 int gms_pipe_create(uint32_t n_buffers, uint64_t buffer_bytes, uint32_t n_readers, gms_pipe **out)
 {

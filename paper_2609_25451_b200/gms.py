@@ -32,7 +32,7 @@ EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
     "gms_verify", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_host_image_alloc", "gms_host_image_free",
-    "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd",
+    "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd", "gms_stage_create", "gms_stage_destroy", "gms_restore_staged",
     "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
     "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
     "gms_launch_geometry", "gms_kernel_launches", "gms_set_device", "gms_strerror", "gms_last_cuda_error", "gms_version",
@@ -87,6 +87,9 @@ def lib():
             "gms_pipe_create": (i, [u32, u64, u32, pp]),
             "gms_pipe_destroy": (i, [p]),
             "gms_restore_fd": (i, [p, p, i, u64, p, p, p, p]),
+            "gms_stage_create": (i, [u32, u64, pp]),
+            "gms_stage_destroy": (i, [p]),
+            "gms_restore_staged": (i, [p, p, p, p, p, p]),
             "gms_service_create": (i, [u64, u32, pp]),
             "gms_service_destroy": (i, [p]),
             "gms_service_acquire_rw": (i, [p]),
@@ -277,6 +280,31 @@ def gms_restore_fd(m: Manifest, pipe: Pipe, fd: int, file_offset: int, d_block_d
     _check(lib().gms_restore_fd(m.handle, pipe.handle, int(fd), int(file_offset), _dev(d_block_digests),
                                 _dev(d_tensor_digests), _stream(stream), C.byref(st)), "gms_restore_fd")
     return {k: getattr(st, k) for k, _ in PipeStats._fields_}
+
+
+class Stage:
+    """Owner of a ``gms_stage*`` (device staging ring fed by the copy engine)."""
+
+    def __init__(self, handle):
+        self.handle = handle
+
+    def close(self):
+        if self.handle:
+            lib().gms_stage_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+
+def gms_stage_create(n_buffers: int, buffer_bytes: int) -> Stage:
+    out = C.c_void_p()
+    _check(lib().gms_stage_create(n_buffers, int(buffer_bytes), C.byref(out)), "gms_stage_create")
+    return Stage(out.value)
+
+
+def gms_restore_staged(m: Manifest, stage: Stage, host_image, d_block_digests, d_tensor_digests, stream=None):
+    _check(lib().gms_restore_staged(m.handle, stage.handle, _dev(host_image), _dev(d_block_digests), _dev(d_tensor_digests),
+                                    _stream(stream)), "gms_restore_staged")
 
 
 STATE_EMPTY, STATE_RW, STATE_COMMITTED, STATE_RO = 0, 1, 2, 3

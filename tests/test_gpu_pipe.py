@@ -67,6 +67,51 @@ def test_restore_fd_equals_restore_of_the_same_bytes(oracle, tmp_path, n_buffers
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("n_buffers,buffer_mib", [(2, 1), (3, 4), (4, 32)])
+def test_restore_staged_equals_restore_of_the_same_bytes(oracle, n_buffers, buffer_mib):
+    """Copy-engine-fed variant: pinned host image -> device ring -> restore kernel, ordered by stream events only."""
+    from gpu_harness import payload_of
+
+    w = W.mixed_manifest(n_small=1500, n_large=3, large_bytes=(7 << 20) + 40, round16=False, seed=321)
+    image = W.random_bytes_host(w.image_bytes, seed=78)
+    slab_h = np.full(w.slab_bytes, FILL, np.uint8)
+    rc, obd, otd = oracle.restore(oracle_record(oracle, w), image, slab_h)
+    assert rc == 0
+    hptr, _, arr = gms.gms_host_image_alloc(w.image_bytes)
+    arr[:] = image
+    d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    stage = gms.gms_stage_create(n_buffers, buffer_mib << 20)
+    try:
+        for _ in range(3):  # back to back: the ring and its events carry over from call to call
+            d.slab.fill_(FILL)
+            d.reset_outputs()
+            gms.gms_restore_staged(d.m, stage, hptr, d.bd_ptr(), d.td_ptr())
+            torch.cuda.synchronize()
+            assert gms.gms_last_device_status(d.m) == 0
+            assert np.array_equal(d.slab_host(), slab_h), "destination bytes (or guard bands) differ"
+            assert np.array_equal(payload_of(d.bd, d.nb), obd) and np.array_equal(payload_of(d.td, d.nt), otd)
+        # the source must be pinned host memory
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_restore_staged(d.m, stage, d.slab, None, None)
+        assert ei.value.status == gms.ERR_KIND
+    finally:
+        torch.cuda.synchronize()
+        stage.close()
+        d.close()
+        gms.gms_host_image_free(hptr)
+
+
+def test_stage_argument_checks_need_no_gpu():
+    out = ctypes.c_void_p()
+    L = gms.lib()
+    assert L.gms_stage_create(1, 1 << 20, ctypes.byref(out)) == gms.ERR_ARG
+    assert L.gms_stage_create(2, 1000, ctypes.byref(out)) == gms.ERR_ARG
+    assert L.gms_stage_create(2, 1 << 20, None) == gms.ERR_NULL
+    assert L.gms_stage_destroy(None) == gms.OK
+    assert L.gms_restore_staged(None, None, None, None, None, None) == gms.ERR_NULL
+
+
+@pytest.mark.gpu
 def test_restore_fd_reports_a_short_file(tmp_path):
     w = W.pack_layout("short", [3 << 20, 5 << 20, 100], seed=5)
     image = W.random_bytes_host(w.image_bytes, seed=1)
