@@ -186,6 +186,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         payload += e.nbytes;
         if (n_blocks >= 0xffffffffull) return GMS_ERR_RANGE;  // digest slots are indexed with 32 bits on the device
     }
+    gms_manifest *m = nullptr;
     try {
         std::vector<uint32_t> order(n);
         std::iota(order.begin(), order.end(), 0u);
@@ -209,7 +210,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         for (size_t i = 1; i < live.size(); ++i)
             if (entries[live[i - 1]].src_offset + entries[live[i - 1]].nbytes > entries[live[i]].src_offset) sources_disjoint = false;
 
-        gms_manifest *m = new gms_manifest();
+        m = new gms_manifest();
         m->sources_disjoint = sources_disjoint;
         m->entries.assign(entries, entries + n);
         m->image_bytes = image_bytes;
@@ -284,6 +285,10 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         *out = m;
         return GMS_OK;
     } catch (const std::bad_alloc &) {
+        if (m) {
+            if (m->d_tables) cudaFree(m->d_tables);
+            delete m;
+        }
         return GMS_ERR_NOMEM;
     }
 }

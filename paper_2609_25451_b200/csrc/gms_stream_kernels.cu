@@ -41,6 +41,7 @@
 // kWaitLimitNs sets GMS_DEV_TIMEOUT in the status word, drains (bounded) what
 // it has in flight and returns.
 #include <algorithm>
+#include <mutex>
 
 #include "gms_internal.h"
 
@@ -205,17 +206,20 @@ struct ListProvider {
     {
         if (lane == 0) raw_next = atomicAdd(counters + home * kCounterStride, 1u);
     }
-    // Counter c hands out chunk runs c, c + n_counters, c + 2 n_counters, ... (a run = `group` consecutive chunks);
-    // warps are spread over the counters,
-    // so the chunks in flight stay a compact moving front of the work list while no single address takes all
-    // the atomics.  A warp whose counter has run dry moves on to the next one (that is the load balancing).
-    // The ticket used here was drawn one step earlier; the next one is drawn now and read a chunk later.
+    // Counter c hands out chunk runs c, c + n_counters, c + 2 n_counters, ... (a run = `group` consecutive
+    // chunks); warps are spread over the counters, so the chunks in flight stay a compact moving front of the
+    // work list while no single address takes all the atomics.  A warp whose counter has run dry moves on to
+    // the next one (that is the load balancing).  The ticket used here was drawn one step earlier; the next one
+    // is drawn now and read a chunk later.
     __device__ __forceinline__ bool advance(uint32_t lane, uint32_t &idx_out)
     {
         if (grp_left) {  // still inside the run of `group` consecutive chunks the last ticket bought
             --grp_left;
-            idx_out = ++grp_idx;
-            return grp_idx < n_chunks;
+            if (++grp_idx < n_chunks) {
+                idx_out = grp_idx;
+                return true;
+            }
+            grp_left = 0;  // the run ran off the end of the list: go and draw elsewhere
         }
         for (;;) {
             const uint32_t t = __shfl_sync(kFull, raw_next, 0);
@@ -614,6 +618,8 @@ cudaError_t get_geometry(Kind kind, Geometry *out)
     cudaError_t e = cudaGetDevice(&dev);
     if (e) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    static std::mutex mu;  // the table is filled once per (device, kernel); callers may come from several threads
+    std::lock_guard<std::mutex> lock(mu);
     if (!g_geom_ok[dev][kind]) {
         int sms = 0, max_smem = 0;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev))) return e;
