@@ -138,7 +138,8 @@ __device__ __forceinline__ uint64_t mix_full(uint64_t z)
 // mix(w ^ c) without its last xor-shift; cfold = c ^ (c >> 30).
 __device__ __forceinline__ uint64_t mix_head(uint64_t w, uint64_t cfold)
 {
-    // (spelling the products on 32-bit halves with mul.hi executes 5 % fewer instructions but runs 7 % slower)
+    // (two hand-spelled 32-bit versions of this -- products via mul.hi, or via mul.wide with explicit funnel shifts --
+    // executed 2-5 % fewer instructions and ran 4-9 % slower; the compiler's own lowering of the 64-bit form stays)
     uint64_t z = (w ^ (w >> 30) ^ cfold) * kM1;
     z = (z ^ (z >> 27)) * kM2;
     return z;
