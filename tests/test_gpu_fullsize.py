@@ -88,6 +88,37 @@ def test_llama3_8b_manifest_full_size(oracle):
     d.close()
 
 
+def test_single_tensor_beyond_4_gib(oracle):
+    """One tensor of 4 GiB + 4 KiB + 1 bytes (more than 2^20 blocks, byte offsets beyond 32 bits, ragged tail):
+    every byte on the device, the whole tensor digest and sampled block digests against the oracle."""
+    n = (4 << 30) + 4096 + 1
+    w = W.pack_layout("huge", [48, n, 16], seed=6)
+    image = torch.empty(w.image_bytes, dtype=torch.uint8, device="cuda")
+    W.fill_random_device(image, 995)
+    d = DeviceWorkload(w, image_dev=image)
+    bd, td = d.restore()
+    assert torch.equal(d.slab, expected_slab(w, image))
+    bd2, td2 = d.digest()
+    assert np.array_equal(bd, bd2) and np.array_equal(td, td2)
+    rec = oracle_record(oracle, w)
+    base, total = oracle.block_bases(rec)
+    assert total == 1 + (1 << 20) + 2 + 1
+    s = int(w.rows[1]["src_offset"])
+    T, obd = oracle.tensor_digest(image[s:s + n].cpu().numpy())  # ~3 s of oracle time
+    assert int(td[1]) == T
+    assert np.array_equal(bd[int(base[1]):int(base[1]) + obd.size], obd)
+    for t in (0, 2):
+        s0, n0 = int(w.rows[t]["src_offset"]), int(w.rows[t]["nbytes"])
+        T0, _ = oracle.tensor_digest(image[s0:s0 + n0].cpu().numpy())
+        assert int(td[t]) == T0
+    # a flip in the very last byte (offset 2^32 + 4096) is named with its block index 2^20 + 1
+    gms.gms_manifest_set_expected(d.m, d.bd_ptr())
+    d.flip(1, n - 1, 7)
+    d.digest()
+    assert d.verify(cap=4) == (1, [(int(w.rows[1]["tensor_id"]), (1 << 20) + 1)])
+    d.close()
+
+
 @pytest.mark.parametrize("round16", [True, False])
 def test_mixed_manifest_full_size_against_the_oracle_in_full(oracle, round16):
     w = W.mixed_manifest(round16=round16)
