@@ -226,6 +226,7 @@ int gms_verify_flat_noalloc(const uint64_t *d_computed, const uint64_t *d_expect
 int gms_last_device_status(const gms_manifest *m, void *stream, uint64_t *word);
 
 /* A paged KV pool: n_planes planes (layer x {K,V}) of n_blocks blocks. */
+#define GMS_KV_IMAGE_BY_ID 1u
 typedef struct {
     void *base;            /* (device) 16-byte aligned                                        */
     uint64_t plane_stride; /* bytes between planes, multiple of 16                            */
@@ -233,7 +234,9 @@ typedef struct {
     uint32_t n_planes;
     uint32_t n_blocks;
     uint32_t block_bytes;  /* multiple of 4096, at most 131072                                */
-    uint32_t reserved;     /* 0                                                               */
+    uint32_t flags;        /* 0, or GMS_KV_IMAGE_BY_ID: the image is pool-shaped -- its slot for
+                              list position j is slot d_block_ids[j] (a subset copy between two
+                              pools of the same shape) instead of slot j (a packed image)        */
 } gms_kv_pool;
 
 /*

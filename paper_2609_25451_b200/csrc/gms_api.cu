@@ -460,6 +460,7 @@ static int kv_call(const gms_kv_pool *pool, const void *image, uint64_t img_plan
          img_plane_stride | img_slot_stride) & 15u)
         return GMS_ERR_ALIGN;
     if (pool->block_stride < pool->block_bytes && pool->n_blocks > 1) return GMS_ERR_ARG;
+    if (pool->flags & ~GMS_KV_IMAGE_BY_ID) return GMS_ERR_ARG;
     const uint64_t k = pool->block_bytes / gms::kBlockBytes;
     if ((uint64_t)n_sel * pool->n_planes * k >= 0xffffffffull) return GMS_ERR_RANGE;
     if (work) {
@@ -483,6 +484,7 @@ static int kv_call(const gms_kv_pool *pool, const void *image, uint64_t img_plan
     a.status = reinterpret_cast<unsigned long long *>(d_status);
     a.hints = 0;
     a.capture = capture ? 1u : 0u;
+    a.by_id = (pool->flags & GMS_KV_IMAGE_BY_ID) ? 1u : 0u;
     GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
 }

@@ -70,6 +70,7 @@ struct KvArgs {
     uint64_t *kv_digests;          // may be null
     unsigned long long *status;    // [0] skipped ids, [1] device status word, [2] work counter, [3] spare
     uint32_t capture;              // 1: gather pool blocks into the image
+    uint32_t by_id;                // 1: the image is pool-shaped (slot = block id), else packed (slot = list position)
     uint32_t hints;                // filled in by the launcher
 };
 

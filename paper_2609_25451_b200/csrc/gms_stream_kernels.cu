@@ -308,7 +308,8 @@ struct KvProvider {
                 if (p == 0 && lane == 0) atomicAdd(a.status, 1ull);
                 continue;
             }
-            uint8_t *img = const_cast<uint8_t *>(a.image) + (uint64_t)p * a.img_plane_stride + (uint64_t)j * a.img_slot_stride;
+            const uint32_t img_slot = a.by_id ? (uint32_t)id : j;  // pool-shaped image: slot = block id
+            uint8_t *img = const_cast<uint8_t *>(a.image) + (uint64_t)p * a.img_plane_stride + (uint64_t)img_slot * a.img_slot_stride;
             uint8_t *blk = a.pool_base + (uint64_t)p * a.plane_stride + (uint64_t)id * a.block_stride;
             it.src = a.capture ? blk : img;
             it.dst = a.capture ? img : blk;

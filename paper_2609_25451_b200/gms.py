@@ -50,7 +50,10 @@ class GmsError(RuntimeError):
 
 class KvPool(C.Structure):
     _fields_ = [("base", C.c_void_p), ("plane_stride", C.c_uint64), ("block_stride", C.c_uint64),
-                ("n_planes", C.c_uint32), ("n_blocks", C.c_uint32), ("block_bytes", C.c_uint32), ("reserved", C.c_uint32)]
+                ("n_planes", C.c_uint32), ("n_blocks", C.c_uint32), ("block_bytes", C.c_uint32), ("flags", C.c_uint32)]
+
+
+KV_IMAGE_BY_ID = 1
 
 
 _lib = None

@@ -126,6 +126,54 @@ def test_kv_capture_parity(oracle):
 
 
 @pytest.mark.gpu
+def test_kv_pool_shaped_image_is_a_subset_copy_between_pools(oracle):
+    """GMS_KV_IMAGE_BY_ID: the image has the pool's shape, so list position j addresses image slot ids[j].  The
+    oracle knows packed images only; the packed image it is given is the pool-shaped one gathered by plain indexing."""
+    rng = np.random.default_rng(91)
+    n_planes, n_blocks, bb = 4, 120, 32768
+    k = bb // 4096
+    ids = rng.permutation(n_blocks)[:45].astype(np.int32)
+    ids[5], ids[20] = -7, n_blocks  # skipped
+    n_sel = len(ids)
+    plane = n_blocks * bb
+    a_h = W.random_bytes_host(n_planes * plane, 401)  # pool A: the "image"
+    b_h = W.random_bytes_host(n_planes * plane, 402)  # pool B: the destination
+    a4 = a_h.reshape(n_planes, n_blocks, bb)
+    packed = np.zeros((n_planes, n_sel, bb), np.uint8)
+    for j, i in enumerate(ids):
+        if 0 <= i < n_blocks:
+            packed[:, j] = a4[:, i]
+    want_b = b_h.copy()
+    rc, obd, okd, oskip = oracle.kv_restore(want_b, plane, bb, n_planes, n_blocks, bb, packed.reshape(-1), n_sel * bb, bb, ids)
+    assert rc == 0 and oskip == 2
+    a_d, b_d = torch.from_numpy(a_h).cuda(), torch.from_numpy(b_h).cuda()
+    ids_d = torch.from_numpy(ids).cuda()
+    bd, kd, st = guarded_u64(n_sel * n_planes * k), guarded_u64(n_sel), guarded_u64(4)
+    desc = gms.KvPool(base=b_d.data_ptr(), plane_stride=plane, block_stride=bb, n_planes=n_planes, n_blocks=n_blocks,
+                      block_bytes=bb, flags=gms.KV_IMAGE_BY_ID)
+    gms.gms_kv_restore(desc, a_d, plane, bb, gms.SRC_DEVICE, ids_d, n_sel, bd.data_ptr() + 8 * PAD, kd.data_ptr() + 8 * PAD,
+                       st.data_ptr() + 8 * PAD)
+    torch.cuda.synchronize()
+    assert payload_of(st, 4)[:2].tolist() == [2, 0]
+    assert np.array_equal(b_d.cpu().numpy(), want_b) and np.array_equal(a_d.cpu().numpy(), a_h)
+    assert np.array_equal(payload_of(bd, n_sel * n_planes * k), obd) and np.array_equal(payload_of(kd, n_sel), okd)
+    # and back: capture B's selected blocks into a third pool-shaped buffer; only those blocks change
+    c_d = torch.full((n_planes * plane,), 0x5C, dtype=torch.uint8, device="cuda")
+    gms.gms_kv_capture(desc, c_d, plane, bb, gms.SRC_DEVICE, ids_d, n_sel, None, kd.data_ptr() + 8 * PAD, st.data_ptr() + 8 * PAD)
+    torch.cuda.synchronize()
+    want_c = np.full((n_planes, n_blocks, bb), 0x5C, np.uint8)
+    for i in ids:
+        if 0 <= i < n_blocks:
+            want_c[:, i] = want_b.reshape(n_planes, n_blocks, bb)[:, i]
+    assert np.array_equal(c_d.cpu().numpy(), want_c.reshape(-1)) and np.array_equal(payload_of(kd, n_sel), okd)
+    bad = gms.KvPool(base=b_d.data_ptr(), plane_stride=plane, block_stride=bb, n_planes=n_planes, n_blocks=n_blocks,
+                     block_bytes=bb, flags=0x10)
+    with pytest.raises(gms.GmsError) as ei:
+        gms.gms_kv_restore(bad, a_d, plane, bb, gms.SRC_DEVICE, ids_d, n_sel, None, None, st.data_ptr() + 8 * PAD)
+    assert ei.value.status == gms.ERR_ARG
+
+
+@pytest.mark.gpu
 def test_capture_full_size_8b_round_trip(oracle):
     """At the benchmark's size: capture the 16 GB of allocations into an image, then check every image byte with
     torch, sampled block digests with the oracle, and that the digests equal those of digest-in-place."""
