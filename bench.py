@@ -397,9 +397,33 @@ def cpu_baseline(args, bench, W, torch):
     assert bad == 0
     nb = int(sum((int(r[3]) + 4095) // 4096 for r in rec))
     traffic = 3 * used + 16 * nb + 2 * 16 * nb
-    return {"value": traffic / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"first {n} tensors of the manifest ({used} B payload), one step = digest+verify+restore+verify, "
-                      f"{dt:.2f} s on 1 of {os.cpu_count()} host cores"}
+    out = {"value": traffic / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"first {n} tensors of the manifest ({used} B payload), one step = digest+verify+restore+verify, "
+                     f"{dt:.2f} s on 1 of {os.cpu_count()} host cores"}
+    # the same oracle functions on all host cores: the sample's tensors are dealt out to threads (the oracle itself
+    # is single-threaded and untouched; ctypes releases the GIL), each thread works on its own sub-record
+    import concurrent.futures as cf
+
+    cores = os.cpu_count() or 1
+    order = sorted(range(len(rec)), key=lambda i: -int(rec[i]["nbytes"]))
+    loads, groups = [0] * cores, [[] for _ in range(cores)]
+    for i in order:  # largest first onto the least loaded thread
+        k = loads.index(min(loads))
+        groups[k].append(i)
+        loads[k] += int(rec[i]["nbytes"])
+    shards = []
+    for g in groups:
+        if g:
+            sub = rec[sorted(g)]
+            _, exp_sub, _ = oracle.digest(sub, slab)  # slab holds the restored bytes: these are the recorded digests
+            shards.append((sub, exp_sub))
+    with cf.ThreadPoolExecutor(len(shards)) as ex:
+        t = time.perf_counter()
+        bad = sum(ex.map(lambda s: oracle_step(oracle, s[0], image, slab, s[1]), shards))
+        dt_all = time.perf_counter() - t
+    assert bad == 0
+    out["all_cores"] = {"value": traffic / dt_all / 1e9, "unit": UNIT, "cores": len(shards), "seconds": dt_all}
+    return out
 
 
 def reference_arm(args):
