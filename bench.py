@@ -104,7 +104,12 @@ class ClockSampler:
                     reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                 except Exception:
                     reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
-                self.samples.append((time.perf_counter(), mhz, reasons))
+                try:
+                    mem = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_MEM)
+                    watts = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                except Exception:
+                    mem, watts = None, None
+                self.samples.append((time.perf_counter(), mhz, reasons, mem, watts))
             except Exception:
                 pass
             time.sleep(0.004)
@@ -138,6 +143,8 @@ class ClockSampler:
         return {
             "sm_mhz": statistics.median(s[1] for s in inside) if inside else None,
             "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(inside), "window": window,
+            "mem_mhz": statistics.median(s[3] for s in inside) if inside and inside[0][3] is not None else None,
+            "power_w": statistics.median(s[4] for s in inside) if inside and inside[0][4] is not None else None,
         }
 
 
