@@ -33,6 +33,7 @@ __device__ __forceinline__ uint32_t diff_mask(const uint64_t *c, const uint64_t 
 
 __global__ void __launch_bounds__(kThreads) gms_verify_count_kernel(VerifyArgs a)
 {
+    asm volatile("griddepcontrol.launch_dependents;");  // the scan kernel may be scheduled; it waits for our counts
     __shared__ uint32_t warp_sum[kThreads / 32];
     const uint64_t first = (uint64_t)blockIdx.x * kVerifySegBlocks + (uint64_t)threadIdx.x * kPerThread;
     uint32_t c = __popc(diff_mask(a.computed, a.expected, first, a.n_blocks));
@@ -51,6 +52,8 @@ __global__ void __launch_bounds__(1024) gms_verify_scan_kernel(VerifyArgs a)
 {
     __shared__ uint64_t warp_tot[32];
     __shared__ uint64_t carry;
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the per-segment counts are complete and visible
     if (threadIdx.x == 0) carry = 0;
     __syncthreads();
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -77,6 +80,7 @@ __global__ void __launch_bounds__(1024) gms_verify_scan_kernel(VerifyArgs a)
 
 __global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // counts (first pass) and offsets (scan) are complete
     if (a.seg_count[blockIdx.x] == 0) return;  // the common case: nothing differs here
     __shared__ uint32_t warp_sum[kThreads / 32];
     const uint64_t first = (uint64_t)blockIdx.x * kVerifySegBlocks + (uint64_t)threadIdx.x * kPerThread;
@@ -177,11 +181,23 @@ cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
     gms_verify_count_kernel<<<a.n_segments, kThreads, 0, s>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e) return e;
-    gms_verify_scan_kernel<<<1, 1024, 0, s>>>(a);
-    if ((e = cudaGetLastError())) return e;
-    gms_verify_emit_kernel<<<a.n_segments, kThreads, 0, s>>>(a);
+    // scan and emit are scheduled while their predecessor still runs (programmatic dependent launch); each
+    // waits for the predecessor's results before reading them
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(1024);
+    if ((e = cudaLaunchKernelEx(&cfg, gms_verify_scan_kernel, a))) return e;
+    cfg.gridDim = dim3(a.n_segments);
+    cfg.blockDim = dim3(kThreads);
+    e = cudaLaunchKernelEx(&cfg, gms_verify_emit_kernel, a);
     count_launches(3);
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s)
