@@ -192,6 +192,14 @@ int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_misma
                uint64_t *d_count, void *stream);
 
 /*
+ * gms_verify_tensors -- the per-tensor summary of the same trust decision (Section 2.2): which
+ * tensors may be reused as they are.  d_tensor_counts (device, n u32, entry order) receives for
+ * every entry the number of its blocks whose digest differs from the recorded one (0 = intact).
+ * Errors: NULL, STATE (nothing recorded), CUDA.
+ */
+int gms_verify_tensors(const gms_manifest *m, const uint64_t *d_block_digests, uint32_t *d_tensor_counts, void *stream);
+
+/*
  * gms_verify_flat_noalloc -- the paper has no counterpart; this is a convenience of this library.
  *
  * Who it is for.  Some callers of a memory service cannot allocate device memory at the moment

@@ -435,6 +435,21 @@ int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_misma
     return GMS_OK;
 }
 
+int gms_verify_tensors(const gms_manifest *m, const uint64_t *d_block_digests, uint32_t *d_tensor_counts, void *stream)
+{
+    if (!m || (m->n_blocks && !d_block_digests) || (!m->entries.empty() && !d_tensor_counts)) return GMS_ERR_NULL;
+    if (m->host_only || !m->has_expected) return GMS_ERR_STATE;
+    gms::VerifyArgs a = {};
+    a.computed = d_block_digests;
+    a.expected = m->d_expected;
+    a.n_blocks = m->n_blocks;
+    a.block_base = m->d_block_base;
+    a.tensor_ids = m->d_tensor_ids;
+    a.n_tensors = (uint32_t)m->entries.size();
+    GMS_CUDA(gms::launch_verify_tensor_counts(a, d_tensor_counts, static_cast<cudaStream_t>(stream)));
+    return GMS_OK;
+}
+
 int gms_last_device_status(const gms_manifest *m, void *stream, uint64_t *word)
 {
     if (!m || !word) return GMS_ERR_NULL;

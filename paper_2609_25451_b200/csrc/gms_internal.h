@@ -93,6 +93,7 @@ struct VerifyArgs {
 };
 constexpr uint32_t kVerifySegBlocks = 2048;  // digest slots compared by one CTA
 cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s);
+cudaError_t launch_verify_tensor_counts(const VerifyArgs &a, uint32_t *counts, cudaStream_t s);
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s);
 
 // A window of a restore that is fed piecewise (file -> pinned buffer -> device): a run of the

@@ -200,6 +200,50 @@ cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
     return e;
 }
 
+namespace {
+
+// Per-tensor summary: counts[t] = number of differing blocks of entry t.  One warp per tensor-sized slice
+// would be badly balanced (1 .. 262,144 blocks per tensor), so the slots are walked grid-stride and the rare
+// differing slot looks its tensor up and bumps that counter.
+__global__ void gms_verify_tensor_counts_kernel(VerifyArgs a, uint32_t *counts)
+{
+    const uint64_t step = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t g = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; g < a.n_blocks; g += step) {
+        if (a.computed[g] == a.expected[g]) continue;
+        uint32_t lo = 0, hi = a.n_tensors;
+        while (hi - lo > 1) {
+            const uint32_t mid = lo + (hi - lo) / 2;
+            if (a.block_base[mid] <= g) lo = mid; else hi = mid;
+        }
+        atomicAdd(counts + lo, 1u);
+    }
+}
+
+__global__ void gms_zero_u32_kernel(uint32_t *p, uint64_t n)
+{
+    asm volatile("griddepcontrol.launch_dependents;");
+    const uint64_t step = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += step) p[i] = 0;
+}
+
+}  // namespace
+
+cudaError_t launch_verify_tensor_counts(const VerifyArgs &a, uint32_t *counts, cudaStream_t s)
+{
+    if (a.n_tensors == 0) return cudaSuccess;
+    uint32_t zb = (a.n_tensors + 255) / 256;
+    gms_zero_u32_kernel<<<zb > 592 ? 592 : zb, 256, 0, s>>>(counts, a.n_tensors);
+    cudaError_t e = cudaGetLastError();
+    if (e) return e;
+    count_launches(1);
+    if (a.n_blocks == 0) return cudaSuccess;
+    uint64_t blocks = (a.n_blocks + 1023) / 1024;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    gms_verify_tensor_counts_kernel<<<(uint32_t)blocks, 256, 0, s>>>(a, counts);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s)
 {
     if (n == 0) return cudaSuccess;

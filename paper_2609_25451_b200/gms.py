@@ -31,7 +31,7 @@ MISMATCH_DTYPE = np.dtype([("tensor_id", "<u8"), ("block", "<u8")])
 EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
-    "gms_verify", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_host_image_alloc", "gms_host_image_free",
+    "gms_verify", "gms_verify_tensors", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_host_image_alloc", "gms_host_image_free",
     "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd", "gms_stage_create", "gms_stage_destroy", "gms_restore_staged",
     "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
     "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
@@ -81,6 +81,7 @@ def lib():
             "gms_capture": (i, [p, p, u32, p, p, p]),
             "gms_digest": (i, [p, p, p, p]),
             "gms_verify": (i, [p, p, p, u32, p, p]),
+            "gms_verify_tensors": (i, [p, p, p, p]),
             "gms_verify_flat_noalloc": (i, [p, p, u64, u64, p, u32, p, p]),
             "gms_last_device_status": (i, [p, p, pu64]),
             "gms_kv_restore": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
@@ -212,6 +213,11 @@ def gms_digest(m: Manifest, d_block_digests, d_tensor_digests, stream=None):
 
 def gms_verify(m: Manifest, d_block_digests, d_out, cap: int, d_count, stream=None):
     _check(lib().gms_verify(m.handle, _dev(d_block_digests), _dev(d_out), cap, _dev(d_count), _stream(stream)), "gms_verify")
+
+
+def gms_verify_tensors(m: Manifest, d_block_digests, d_tensor_counts, stream=None):
+    _check(lib().gms_verify_tensors(m.handle, _dev(d_block_digests), _dev(d_tensor_counts), _stream(stream)),
+           "gms_verify_tensors")
 
 
 def gms_verify_flat_noalloc(d_computed, d_expected, n_blocks: int, tensor_id: int, d_out, cap: int, d_count, stream=None):

@@ -157,6 +157,14 @@ def test_many_mismatches_exceed_cap_in_order(oracle, scale):
         ocount, omm = oracle.verify(rec, obd, want_bd, cap=cap)
         assert count == ocount and count > 2500
         assert pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+    # per-tensor summary = the oracle's full mismatch list counted per tensor id (entry order)
+    ocount, omm = oracle.verify(rec, obd, want_bd, cap=1 << 20)
+    want_counts = [sum(1 for m in omm if int(m["tensor_id"]) == int(r["tensor_id"])) for r in w.rows]
+    tc = torch.full((len(w.rows) + 2,), 0x7777, dtype=torch.int32, device="cuda")
+    gms.gms_verify_tensors(d.m, d.bd_ptr(), tc.data_ptr() + 4)
+    torch.cuda.synchronize()
+    got = tc.cpu().tolist()
+    assert got[0] == 0x7777 and got[-1] == 0x7777 and got[1:-1] == want_counts and sum(want_counts) == ocount
     d.close()
 
 
