@@ -120,7 +120,12 @@ int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vect
             return e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : cuda_fail(e);
         }
         e = cudaMemcpy(m->d_by_src, m->by_src.data(), m->by_src.size() * sizeof(Chunk), cudaMemcpyHostToDevice);
-        if (e != cudaSuccess) return cuda_fail(e);
+        if (e != cudaSuccess) {
+            cudaFree(m->d_by_src);
+            m->d_by_src = nullptr;
+            m->by_src.clear();
+            return cuda_fail(e);
+        }
     }
     out->clear();
     size_t i = 0;
@@ -225,8 +230,8 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         }
         m->block_base[n] = acc;
 
-        // ---- chunk size: small enough that every warp of the grid gets several chunks
-        uint32_t total_warps = 148 * 12;
+        // ---- chunk length (needs the number of warps the restore kernel runs; a B200's if no device is asked)
+        uint32_t total_warps = 148 * 8;
         if (!m->host_only) {
             gms::Geometry g;
             cudaError_t e = gms::get_geometry(gms::kRestore, &g);
