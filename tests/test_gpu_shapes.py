@@ -39,6 +39,13 @@ def test_parity_in_other_launch_shapes(env):
     assert r.returncode == 0 and r.stdout.strip().startswith("OK"), r.stdout[-2000:] + r.stderr[-4000:]
 
 
+def test_short_randomised_soak():
+    """Ten seconds of tests/fuzz_parity.py (random manifests, operations, corruption, KV lists) against the oracle."""
+    r = subprocess.run([sys.executable, os.path.join(HERE, "fuzz_parity.py"), "--seconds", "10", "--seed", "7"],
+                       capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "FUZZ OK" in r.stdout, r.stdout[-2000:] + r.stderr[-4000:]
+
+
 def test_image_base_only_16_byte_aligned(oracle):
     w = W.mixed_manifest(n_small=700, n_large=1, large_bytes=(3 << 20) + 8, round16=False, seed=55)
     image = W.random_bytes_host(w.image_bytes, seed=6)
