@@ -35,8 +35,23 @@ __global__ void __launch_bounds__(kThreads) gms_verify_count_kernel(VerifyArgs a
 {
     asm volatile("griddepcontrol.launch_dependents;");  // the scan kernel may be scheduled; it waits for our counts
     __shared__ uint32_t warp_sum[kThreads / 32];
-    const uint64_t first = (uint64_t)blockIdx.x * kVerifySegBlocks + (uint64_t)threadIdx.x * kPerThread;
-    uint32_t c = __popc(diff_mask(a.computed, a.expected, first, a.n_blocks));
+    // only the segment's total matters here, so the slots are read coalesced (16-byte pairs, neighbouring lanes
+    // neighbouring pairs); the emit pass, which needs ranks, uses the thread-contiguous layout
+    const uint64_t seg0 = (uint64_t)blockIdx.x * kVerifySegBlocks;
+    const bool vec = ((reinterpret_cast<uint64_t>(a.computed) | reinterpret_cast<uint64_t>(a.expected)) & 15u) == 0;
+    uint32_t c = 0;
+#pragma unroll
+    for (uint32_t k = 0; k < kPerThread / 2; ++k) {
+        const uint64_t g = seg0 + 2ull * (k * kThreads + threadIdx.x);
+        if (vec && g + 1 < a.n_blocks) {
+            const ulonglong2 p = *reinterpret_cast<const ulonglong2 *>(a.computed + g);
+            const ulonglong2 q = *reinterpret_cast<const ulonglong2 *>(a.expected + g);
+            c += (p.x != q.x) + (p.y != q.y);
+        } else {  // arrays that are only 8-byte aligned, and the odd last slot
+            if (g < a.n_blocks) c += a.computed[g] != a.expected[g];
+            if (g + 1 < a.n_blocks) c += a.computed[g + 1] != a.expected[g + 1];
+        }
+    }
     c = __reduce_add_sync(0xffffffffu, c);
     if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = c;
     __syncthreads();

@@ -157,6 +157,16 @@ def test_many_mismatches_exceed_cap_in_order(oracle, scale):
         ocount, omm = oracle.verify(rec, obd, want_bd, cap=cap)
         assert count == ocount and count > 2500
         assert pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+    # the computed digests may sit at an address that is only 8-byte aligned
+    shifted = torch.zeros(d.nb + 1, dtype=torch.int64, device="cuda")
+    shifted[1:] = d.bd[PAD:PAD + d.nb]
+    out = torch.zeros(2 * 16, dtype=torch.int64, device="cuda")
+    cnt = torch.zeros(1, dtype=torch.int64, device="cuda")
+    gms.gms_verify(d.m, shifted.data_ptr() + 8, out, 16, cnt)
+    torch.cuda.synchronize()
+    ocount, omm = oracle.verify(rec, obd, want_bd, cap=16)
+    assert int(cnt.item()) == ocount
+    assert out.cpu().numpy().view(np.uint64).reshape(16, 2).tolist() == [[int(m["tensor_id"]), int(m["block"])] for m in omm]
     # per-tensor summary = the oracle's full mismatch list counted per tensor id (entry order)
     ocount, omm = oracle.verify(rec, obd, want_bd, cap=1 << 20)
     want_counts = [sum(1 for m in omm if int(m["tensor_id"]) == int(r["tensor_id"])) for r in w.rows]
