@@ -88,6 +88,69 @@ def test_llama3_8b_manifest_full_size(oracle):
     d.close()
 
 
+def test_llama3_8b_manifest_fed_from_a_file_and_from_a_pinned_image(oracle, tmp_path):
+    """The 16 GB manifest restored twice more without a resident device image: through gms_restore_fd (file ->
+    pinned ring -> kernel) and gms_restore_staged (pinned image -> copy engine -> device ring -> kernel).  Both must
+    leave exactly the bytes and digests of the plain device-staged restore; sampled blocks are checked with the oracle."""
+    import os
+    import shutil
+
+    w = W.llama3_8b_manifest()
+    shm = "/dev/shm" if os.path.isdir("/dev/shm") and shutil.disk_usage("/dev/shm").free > w.image_bytes + (2 << 30) else None
+    if shm is None and shutil.disk_usage(str(tmp_path)).free < w.image_bytes + (2 << 30):
+        pytest.skip("no room for a 16 GB snapshot file")
+    try:
+        hptr, _, arr = gms.gms_host_image_alloc(w.image_bytes)
+    except gms.GmsError as e:
+        pytest.skip(f"cannot pin 16 GB of host memory here: {e}")
+    path = os.path.join(shm or str(tmp_path), f"gms_test_image_{os.getpid()}.bin")
+    try:
+        image = torch.empty(w.image_bytes, dtype=torch.uint8, device="cuda")
+        W.fill_random_device(image, 996)
+        cpu = torch.from_numpy(arr)
+        for a in range(0, w.image_bytes, 1 << 30):
+            cpu[a:a + (1 << 30)].copy_(image[a:a + (1 << 30)])
+        with open(path, "wb") as f:
+            for a in range(0, w.image_bytes, 1 << 30):
+                f.write(arr[a:a + (1 << 30)].tobytes())
+        d = DeviceWorkload(w, image_dev=image)
+        bd, td = d.restore()
+        want = d.slab.clone()
+        rec = oracle_record(oracle, w)
+        base, _ = oracle.block_bases(rec)
+        check_sampled_blocks(oracle, w, image, bd, base, np.random.default_rng(41), 100)
+        del image
+        d.image = torch.zeros(16, dtype=torch.uint8, device="cuda")  # no device image from here on
+
+        pipe = gms.gms_pipe_create(4, 256 << 20, 16)
+        fd = os.open(path, os.O_RDONLY)
+        d.slab.fill_(FILL)
+        d.reset_outputs()
+        st = gms.gms_restore_fd(d.m, pipe, fd, 0, d.bd_ptr(), d.td_ptr())
+        os.close(fd)
+        pipe.close()
+        from gpu_harness import payload_of
+
+        assert torch.equal(d.slab, want) and st["bytes_read"] <= w.image_bytes
+        assert np.array_equal(payload_of(d.bd, d.nb), bd) and np.array_equal(payload_of(d.td, d.nt), td)
+
+        stage = gms.gms_stage_create(3, 64 << 20)
+        d.slab.fill_(FILL)
+        d.reset_outputs()
+        gms.gms_restore_staged(d.m, stage, hptr, d.bd_ptr(), d.td_ptr())
+        torch.cuda.synchronize()
+        assert torch.equal(d.slab, want)
+        assert np.array_equal(payload_of(d.bd, d.nb), bd) and np.array_equal(payload_of(d.td, d.nt), td)
+        assert gms.gms_last_device_status(d.m) == 0
+        stage.close()
+        d.close()
+    finally:
+        torch.cuda.synchronize()
+        if os.path.exists(path):
+            os.remove(path)
+        gms.gms_host_image_free(hptr)
+
+
 def test_single_tensor_beyond_4_gib(oracle):
     """One tensor of 4 GiB + 4 KiB + 1 bytes (more than 2^20 blocks, byte offsets beyond 32 bits, ragged tail):
     every byte on the device, the whole tensor digest and sampled block digests against the oracle."""
