@@ -91,7 +91,7 @@ extern "C" {
 
 typedef struct gms_manifest gms_manifest; /* opaque */
 
-/* One recorded tensor layout (Section 4: "the client records tensor layouts"). */
+/* One recorded tensor layout (Section 4: what the writing client notes for each tensor before it commits). */
 typedef struct {
     uint64_t tensor_id;  /* caller's identifier, unique within a manifest                     */
     uint64_t src_offset; /* byte offset of the tensor in the packed image, 16-byte aligned    */
