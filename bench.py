@@ -56,6 +56,7 @@ def parse_args():
     ap.add_argument("--vmm", action="store_true", help="8b/mixed/tiny/capture/file: destinations from gms_service VMM slabs")
     ap.add_argument("--graph", action="store_true",
                     help="8b/mixed/tiny: capture the step into a CUDA graph once and time its replays (whole step only)")
+    ap.add_argument("--no-l2-flush", action="store_true", help="mixed/tiny: leave L2 as the previous step left it")
     ap.add_argument("--file-dir", default="/dev/shm", help="file: where the snapshot file is written")
     ap.add_argument("--pipe-buffers", type=int, default=4)
     ap.add_argument("--pipe-mib", type=int, default=256)
@@ -214,6 +215,8 @@ class ManifestBench:
         self.dominant_bytes = self.bytes_restore
         self.launches_per_step = None
         self.graph = None
+        # a working set that L2 (126 MB) could hold between steps is flushed out before every step
+        self.l2_flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev) if self.payload < (512 << 20) else None
 
     def use_graph(self):
         """Captures one step into a CUDA graph; later steps replay it (no per-phase times then)."""
@@ -262,7 +265,9 @@ class ManifestBench:
                             f"{self.m.n_blocks} digest blocks, {self.n_chunks} chunks",
                 "step": "gms_digest + gms_verify + gms_restore(device image) + gms_verify",
                 "destinations": "gms_service VMM slabs (2 GiB, first fit)" if self.vmm else "carved from one cudaMalloc slab",
-                "l2": "inputs larger than L2 (no flush)" if self.payload > (512 << 20) else "working set near L2 size; not flushed",
+                "l2": "inputs larger than L2 (no flush)" if self.payload >= (512 << 20) else
+                      ("L2 flushed before every step (256 MiB read+write, outside the phase events); ms_per_step = sum of phases"
+                       if self.l2_flush is not None else "working set near L2 size; not flushed"),
                 "payload_bytes": self.payload}
 
 
@@ -332,8 +337,15 @@ def event_list(torch, n):
     return [torch.cuda.Event(enable_timing=True) for _ in range(n)]
 
 
+PHASE_STATS = {}  # per-phase median and best of the last timed_steps() call (ms)
+
+
 def timed_steps(torch, bench, steps, dist=None, **step_kw):
-    """Times `steps` steps with CUDA events on the current stream; returns (total ms, per-phase mean ms)."""
+    """Times `steps` steps with CUDA events on the current stream; returns (total ms, per-phase mean ms).
+
+    If the bench object carries an `l2_flush` tensor (working sets that would otherwise sit in L2), it is
+    rewritten before every step, outside every phase's event pair, and the total is the sum of the phases."""
+    flush = getattr(bench, "l2_flush", None)
     n_marks = len(bench.phase_names) + 1
     marks = [event_list(torch, n_marks) for _ in range(steps)]
     e0, e1 = event_list(torch, 2)
@@ -344,6 +356,8 @@ def timed_steps(torch, bench, steps, dist=None, **step_kw):
     t0 = time.perf_counter()
     e0.record()
     for i in range(steps):
+        if flush is not None:
+            flush.add_(1)  # read + write of a buffer twice the size of L2
         bench.step(marks[i], **step_kw)
     e1.record()
     torch.cuda.synchronize()
@@ -353,8 +367,13 @@ def timed_steps(torch, bench, steps, dist=None, **step_kw):
         torch.cuda.synchronize()
     total = e0.elapsed_time(e1)
     phases = {}
+    PHASE_STATS.clear()
     for p, name in enumerate(bench.phase_names):
-        phases[name] = statistics.fmean(marks[i][p].elapsed_time(marks[i][p + 1]) for i in range(steps))
+        ts = [marks[i][p].elapsed_time(marks[i][p + 1]) for i in range(steps)]
+        phases[name] = statistics.fmean(ts)
+        PHASE_STATS[name] = {"median": statistics.median(ts), "best": min(ts)}
+    if flush is not None:
+        total = sum(phases.values()) * steps
     return total, phases, (t0, t1)
 
 
@@ -515,6 +534,38 @@ def host_image_of(torch, gms, dev_image):
     return hptr, dview, cpu
 
 
+def per_tensor_memcpy_yardstick(torch, bench, reps=3):
+    """The launch-per-tensor way of moving the same payload (no digest): one device-to-device cudaMemcpyAsync per
+    manifest entry on one stream, issued through ctypes.  Returns (best device-timed ms, best host-issue ms, calls)."""
+    import ctypes
+
+    try:
+        rt = ctypes.CDLL("libcudart.so.12")  # the runtime torch has already loaded
+    except OSError:
+        return None
+    f = rt.cudaMemcpyAsync
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_void_p]
+    f.restype = ctypes.c_int
+    base = bench.image.data_ptr()
+    e = bench.entries
+    calls = [(int(d), base + int(s), int(n)) for d, s, n in zip(e["dst"], e["src_offset"], e["nbytes"]) if n]
+    stream = torch.cuda.current_stream().cuda_stream
+    best_dev, best_host = float("inf"), float("inf")
+    for _ in range(reps):
+        a, b = event_list(torch, 2)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        a.record()
+        for d, s, n in calls:
+            if f(d, s, n, 3, stream):  # 3 = cudaMemcpyDeviceToDevice
+                return None
+        b.record()
+        t1 = time.perf_counter()
+        torch.cuda.synchronize()
+        best_dev, best_host = min(best_dev, a.elapsed_time(b)), min(best_host, (t1 - t0) * 1e3)
+    return best_dev, best_host, len(calls)
+
+
 def h2d_yardstick(torch, cpu_tensor, dev_tensor, reps=3):
     """Plain cudaMemcpyAsync host->device of the whole pinned image (torch copy_), best of reps, GB/s."""
     best = None
@@ -571,6 +622,8 @@ def main():
         run_file(args, torch, gms, W, dev, sampler, rank)
         return
 
+    if args.no_l2_flush and getattr(bench, "l2_flush", None) is not None:
+        bench.l2_flush = None
     for _ in range(max(args.warmup, 3)):
         bench.step()
     bench.check()
@@ -620,9 +673,16 @@ def main():
         "ms_per_step": max_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u64", "data": "synthetic", "config": bench.config(), "roofline": roofline, "clocks": clocks,
         "gpu_launches": int(launches),
-        "phases_ms": phases,
+        "phases_ms": phases, "phases_ms_median_best": {} if graphed else dict(PHASE_STATS),
         "geometry": gms.gms_launch_geometry(),
     }
+    if type(bench) is ManifestBench and "restore" in phases:
+        y = per_tensor_memcpy_yardstick(torch, bench)
+        if y:
+            line["per_tensor_memcpy"] = {
+                "ms": y[0], "host_issue_ms": y[1], "calls": y[2], "payload_gbs": bench.payload / y[0] / 1e6,
+                "restore_speedup": y[0] / phases["restore"],
+                "note": "one cudaMemcpyAsync D2D per tensor on one stream, no digest (the launch-per-tensor yardstick)"}
     if graphed:
         line["config"]["launch"] = f"CUDA graph replay ({bench.launches_per_step} kernel nodes per step)"
     if "restore" in phases:
