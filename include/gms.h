@@ -6,11 +6,12 @@
  * Memory Lifetime in Dynamo").  Section 3.2 moves model state into device
  * allocations owned by a per-GPU service so that it outlives an engine:
  * a writer populates the allocations and commits them, later engines attach
- * read-only.  Section 4 (GMS paragraph) adds that the client "records tensor
- * layouts" before commit and that, when the service is cold, a separate
- * read-write client repopulates model state in parallel with process restore.
+ * read-only.  Section 4 (GMS paragraph) adds that the writer notes where each
+ * tensor lies before it commits and that, when the service comes up cold, a
+ * fresh writer fills the model state in again while the process is restored.
  * Section 3.1 models the cost of that as S / B_eff, and Section 5.2 observes
- * that today's tool copies device memory serially and leaves the link idle.
+ * that the checkpoint tool in use moves device memory piece by piece, far
+ * below what the link could carry.
  * Section 2.2 allows reuse of surviving allocations only if their contents are
  * intact.  The paper leaves the bulk data path and the integrity check
  * unspecified; this library is that path:
@@ -291,8 +292,8 @@ int gms_host_image_alloc(uint64_t nbytes, void **host_ptr, void **device_view);
 int gms_host_image_free(void *host_ptr);
 
 /*
- * gms_pipe_* / gms_restore_fd -- Section 4, GMS paragraph: with a cold service, a read-write client
- * repopulates model state from storage while the process is being restored; Section 3.1 prices it
+ * gms_pipe_* / gms_restore_fd -- Section 4, GMS paragraph: with a cold service, a fresh writer
+ * fills the model state in from storage while the process is being restored; Section 3.1 prices it
  * at S / B_eff.  The image is read from a file descriptor, never resident as a whole: a ring of
  * `n_buffers` pinned, device-mapped buffers of `buffer_bytes` each (>= 1 MiB, multiple of 4096) is
  * filled by `n_readers` threads with pread(), and each filled buffer is consumed by the restore
@@ -317,7 +318,7 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
 
 /*
  * gms_stage_* / gms_restore_staged -- host-sourced restore with the copy engine on the link
- * (Section 5.2: the existing tool "does not saturate PCIe"; Section 3.1: S / B_eff).  Kernel-issued
+ * (Section 5.2: the existing tool stays far below the PCIe rate; Section 3.1: S / B_eff).  Kernel-issued
  * reads of mapped host memory (gms_restore with GMS_SRC_HOST_MAPPED) top out below what the DMA
  * engine reaches on the same link.  Here the pinned host image is moved window by window with
  * cudaMemcpyAsync on an internal stream into a ring of `n_buffers` device buffers of `buffer_bytes`

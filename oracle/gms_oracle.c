@@ -9,9 +9,9 @@
  *
  * What it states.  The paper (Section 3.2, GMS; Section 3.3, Snapshots with
  * GMS; Section 4, GMS paragraph) describes model state that lives in
- * service-owned device allocations, a client that "records tensor layouts"
- * before commit, a cold-service path in which a read-write client repopulates
- * those allocations, and a warm path in which a replacement engine reuses the
+ * service-owned device allocations, a writer that notes every tensor's place
+ * before it commits, a cold-service path in which a fresh writer fills those
+ * allocations again, and a warm path in which a replacement engine reuses the
  * surviving bytes provided they are still intact (Section 2.2).  The paper
  * gives no digest and no record format; the library fixes both, and this file
  * writes that definition out literally:
