@@ -86,6 +86,13 @@ extern "C" {
 /* gms_manifest_build flags */
 #define GMS_BUILD_HOST_ONLY 1u /* validate and build the work list on the host only (no CUDA
                                   call is made; device entry points return GMS_ERR_STATE)     */
+#define GMS_BUILD_SELFTEST_STALL 2u /* self-test of the bounded waits, for test suites only: in every
+                                  gms_restore / gms_capture / gms_digest of this manifest the barrier of
+                                  the first block of chunk 0 is told to expect 16 bytes that are never
+                                  sent, so the warp that claims it gives up after its wait limit (2 s),
+                                  sets GMS_DEV_TIMEOUT, drains its copies and returns; the other warps
+                                  finish their work.  Nothing faults; outputs of that call are
+                                  incomplete by design.                                        */
 
 /* bits of the device status word */
 #define GMS_DEV_TIMEOUT 1ull   /* a warp gave up waiting for one of its own bulk copies       */
@@ -231,7 +238,8 @@ int gms_verify_tensors(const gms_manifest *m, const uint64_t *d_block_digests, u
 int gms_verify_flat_noalloc(const uint64_t *d_computed, const uint64_t *d_expected, uint64_t n_blocks, uint64_t tensor_id,
                             gms_mismatch *d_out, uint32_t cap, uint64_t *d_count, void *stream);
 
-/* Device status word of the manifest's last call (synchronises `stream`). 0 = clean. */
+/* Device status word of the manifest's last call (synchronises `stream`). 0 = clean; if GMS_DEV_TIMEOUT is
+ * set the word is still stored and the call returns GMS_ERR_TIMEOUT (that call's outputs are incomplete). */
 int gms_last_device_status(const gms_manifest *m, void *stream, uint64_t *word);
 
 /* A paged KV pool: n_planes planes (layer x {K,V}) of n_blocks blocks. */

@@ -23,6 +23,7 @@ struct gms_manifest {
     std::vector<Chunk> chunks;
     uint64_t image_bytes = 0, payload = 0, n_blocks = 0;
     bool host_only = false;
+    bool selftest_stall = false;  // GMS_BUILD_SELFTEST_STALL
     bool sources_disjoint = true;  // image ranges pairwise disjoint (needed by gms_capture only)
     int device = -1;
     // device tables (one allocation) and the recorded digests (allocated on first use)
@@ -164,6 +165,7 @@ int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void
     a.group = 1;
     a.capture = 0;
     a.keep_accum = first ? 0u : 1u;
+    a.stall_chunk = 0xffffffffu;
     cudaError_t e = launch_restore(a, s);
     return e == cudaSuccess ? GMS_OK : cuda_fail(e);
 }
@@ -176,7 +178,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
 {
     if (!out || (n && !entries)) return GMS_ERR_NULL;
     *out = nullptr;
-    if (flags & ~GMS_BUILD_HOST_ONLY) return GMS_ERR_ARG;
+    if (flags & ~(GMS_BUILD_HOST_ONLY | GMS_BUILD_SELFTEST_STALL)) return GMS_ERR_ARG;
     if (n >= 0xffffffffull) return GMS_ERR_RANGE;
 
     // ---- validation (all on the host, before any CUDA call)
@@ -222,6 +224,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         m->payload = payload;
         m->n_blocks = n_blocks;
         m->host_only = (flags & GMS_BUILD_HOST_ONLY) != 0;
+        m->selftest_stall = (flags & GMS_BUILD_SELFTEST_STALL) != 0;
         m->block_base.resize(n + 1);
         uint64_t acc = 0;
         for (size_t t = 0; t < n; ++t) {
@@ -377,6 +380,7 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
     a.group = 1;
     a.capture = capture ? 1u : 0u;
     a.keep_accum = 0;
+    a.stall_chunk = m->selftest_stall ? 0u : 0xffffffffu;
     GMS_CUDA(store ? gms::launch_restore(a, static_cast<cudaStream_t>(stream))
                    : gms::launch_digest(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;

@@ -56,6 +56,7 @@ struct StreamArgs {
     uint32_t group;                // filled in by the launcher
     uint32_t capture;              // 1: gather allocations into the image (restore kernel with roles swapped)
     uint32_t keep_accum;           // 1: a later window of a windowed restore (accumulators and status are kept)
+    uint32_t stall_chunk;          // self-test (GMS_BUILD_SELFTEST_STALL): chunk whose first wait runs out; else 0xffffffff
 };
 
 struct KvArgs {

@@ -58,6 +58,7 @@ struct Item {  // one chunk as the pipeline sees it
     const uint8_t *src;
     uint8_t *dst;
     uint32_t nbytes, tensor, gblock0, tblock0;
+    uint32_t stall;  // self-test only: bytes announced on the first block's barrier that never arrive (else 0)
 };
 
 constexpr uint32_t kFifo = 8;  // chunk records in flight between a warp's issue side and its digest side (>= ring slots)
@@ -195,6 +196,8 @@ struct ListProvider {
     uint32_t group;          // consecutive chunks bought by one ticket
     uint32_t grp_left, grp_idx;
     uint4 da, db;            // buffered descriptor
+    uint32_t buffered;       // its index in the list
+    uint32_t stall_chunk;    // self-test: the chunk whose first wait is made to run out (0xffffffff: none)
     bool have;
 
     __device__ __forceinline__ void load(uint32_t idx)
@@ -202,6 +205,7 @@ struct ListProvider {
         const uint4 *p = reinterpret_cast<const uint4 *>(chunks + idx);
         da = __ldg(p);
         db = __ldg(p + 1);
+        buffered = idx;
     }
     __device__ __forceinline__ void draw(uint32_t lane)
     {
@@ -263,6 +267,7 @@ struct ListProvider {
         it.tensor = db.y;
         it.gblock0 = db.z;
         it.tblock0 = db.w;
+        it.stall = buffered == stall_chunk ? 16u : 0u;
         uint32_t idx;
         have = advance(lane, idx);
         if (have) load(idx);
@@ -317,6 +322,7 @@ struct KvProvider {
             it.tensor = j;
             it.gblock0 = slot0;
             it.tblock0 = p * k;
+            it.stall = 0;
             return true;
         }
         return false;
@@ -406,7 +412,7 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
                 __syncwarp();
             }
             if (lane == 0) {
-                mbar_arrive_expect_tx(bars_s + 8u * s, m16);
+                mbar_arrive_expect_tx(bars_s + 8u * s, m16 + (it_next == 0 ? it.stall : 0u));
                 if (m16) {
                     if (ld_hint)
                         bulk_load_hint(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s, ld_pol);
@@ -520,6 +526,7 @@ __global__ void __launch_bounds__(512, 1) gms_stream_kernel(StreamArgs a)
     prov.group = a.group;
     prov.image = kStore ? a.image : nullptr;
     prov.capture = kStore && a.capture;
+    prov.stall_chunk = a.stall_chunk;
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the prologue's zeroed counters and accumulators are visible from here
     prov.init(threadIdx.x & 31u, blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5));
     run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.hints);

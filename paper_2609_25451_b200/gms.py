@@ -23,6 +23,8 @@ ERR_CUDA, ERR_KIND, ERR_TIMEOUT, ERR_STATE, ERR_ARG, ERR_TOO_LARGE, ERR_IO = -7,
 NOALLOC_MAX_BLOCKS = 4194304
 SRC_DEVICE, SRC_HOST_MAPPED = 0, 1
 BUILD_HOST_ONLY = 1
+BUILD_SELFTEST_STALL = 2  # test suites only: one warp's first wait runs out (see include/gms.h)
+DEV_TIMEOUT = 1  # bit of the device status word
 
 # numpy view of gms_entry / gms_mismatch (32 and 16 bytes)
 ENTRY_DTYPE = np.dtype([("tensor_id", "<u8"), ("src_offset", "<u8"), ("dst", "<u8"), ("nbytes", "<u8")])
