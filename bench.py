@@ -472,6 +472,27 @@ def cpu_baseline(args, bench, W, torch):
     return out
 
 
+def cpu_baseline_kv(bench, planes=16):
+    """The oracle's kv_restore (1 thread) on the first `planes` planes of the same pool shape, image and id list."""
+    import numpy as np
+
+    from oracle import gms_oracle as oracle
+
+    k = bench.k
+    planes = min(planes, k.n_planes)
+    image = bench.image[: planes * k.img_plane_stride].cpu().numpy()
+    pool = np.empty(planes * k.plane_stride, dtype=np.uint8)  # only the selected blocks are ever touched
+    t = time.perf_counter()
+    rc, bd, kd, skipped = oracle.kv_restore(pool, k.plane_stride, k.block_stride, planes, k.n_blocks, k.block_bytes, image,
+                                            k.img_plane_stride, k.img_slot_stride, k.ids)
+    dt = time.perf_counter() - t
+    assert rc == 0 and skipped == 0
+    moved = planes * len(k.ids) * k.block_bytes
+    return {"value": (2 * moved + 8 * bd.size) / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {planes} of {k.n_planes} planes of the same pool, image and id list ({moved} B moved), "
+                      f"{dt:.2f} s on 1 of {os.cpu_count()} host cores"}
+
+
 def reference_arm(args):
     """`--impl reference`: the oracle on this host's cores, same metric, bounded sample per step."""
     rank, _, world = dist_env()
@@ -750,6 +771,8 @@ def main():
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline and type(bench) is ManifestBench:
         line["cpu_baseline"] = cpu_baseline(args, bench, W, torch)
+    elif rank == 0 and world == 1 and not args.no_cpu_baseline and type(bench) is KvBench:
+        line["cpu_baseline"] = cpu_baseline_kv(bench)
 
     if rank == 0:
         print(json.dumps(line), flush=True)
