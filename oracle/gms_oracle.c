@@ -302,3 +302,35 @@ int gmso_kv_capture(const uint8_t *pool_base, uint64_t plane_stride, uint64_t bl
     if (skipped) *skipped = skip;
     return GMSO_OK;
 }
+
+/*
+ * Paged-KV subset digest in place: the check that decides whether KV blocks that outlived an engine may be reused
+ * (Section 6, "Preserving KV state", read together with Section 2.2: surviving state is reused only if intact).
+ * Pool block ids[j] of every plane is digested where it lies; nothing is written to the pool.  Digests are laid
+ * out exactly as in gmso_kv_restore.  An id outside [0, n_blocks) is skipped: digests 0, *skipped incremented.
+ */
+int gmso_kv_digest(const uint8_t *pool_base, uint64_t plane_stride, uint64_t block_stride, uint32_t n_planes,
+                   uint32_t n_blocks, uint32_t block_bytes, const int32_t *ids, uint32_t n_sel, uint64_t *block_digests,
+                   uint64_t *kv_digests, uint64_t *skipped)
+{
+    uint64_t k = block_bytes / GMSO_BLOCK, skip = 0;
+    if (block_bytes == 0 || block_bytes % GMSO_BLOCK) return GMSO_ERR_ALIGN;
+    if (n_sel && (!pool_base || !ids)) return GMSO_ERR_NULL;
+    for (uint32_t j = 0; j < n_sel; ++j) {
+        int ok = ids[j] >= 0 && (uint32_t)ids[j] < n_blocks;
+        uint64_t K = 0;
+        if (!ok) ++skip;
+        for (uint32_t p = 0; p < n_planes; ++p) {
+            const uint8_t *blk = ok ? pool_base + (uint64_t)p * plane_stride + (uint64_t)ids[j] * block_stride : NULL;
+            for (uint64_t c = 0; c < k; ++c) {
+                uint64_t q = (uint64_t)p * k + c;
+                uint64_t d = ok ? gmso_block_digest(blk + c * GMSO_BLOCK, GMSO_BLOCK) : 0;
+                if (block_digests) block_digests[((uint64_t)j * n_planes + p) * k + c] = d;
+                if (ok) K ^= gmso_mix(d ^ (q * GMSO_G));
+            }
+        }
+        if (kv_digests) kv_digests[j] = ok ? K : 0;
+    }
+    if (skipped) *skipped = skip;
+    return GMSO_OK;
+}

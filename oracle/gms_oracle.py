@@ -69,6 +69,8 @@ def lib():
         L.gmso_digest.argtypes = [p, C.c_size_t, p, u64, p, p]
         L.gmso_verify.restype = u64
         L.gmso_verify.argtypes = [p, C.c_size_t, p, p, p, u64]
+        L.gmso_kv_digest.restype = C.c_int
+        L.gmso_kv_digest.argtypes = [p, u64, u64, C.c_uint32, C.c_uint32, C.c_uint32, p, C.c_uint32, p, p, p]
         L.gmso_kv_restore.restype = C.c_int
         L.gmso_kv_restore.argtypes = [p, u64, u64, C.c_uint32, C.c_uint32, C.c_uint32, p, u64, u64, p, C.c_uint32, p, p, p]
         _lib = L
@@ -213,4 +215,21 @@ def kv_capture(pool: np.ndarray, plane_stride: int, block_stride: int, n_planes:
     rc = lib().gmso_kv_capture(_ptr(pool_b), plane_stride, block_stride, n_planes, n_blocks, block_bytes, _ptr(img),
                                img_plane_stride, img_slot_stride, _ptr(ids), len(ids), _ptr(bd), _ptr(kd),
                                C.addressof(skipped))
+    return int(rc), bd, kd, int(skipped.value)
+
+
+def kv_digest(pool: np.ndarray, plane_stride: int, block_stride: int, n_planes: int, n_blocks: int,
+              block_bytes: int, ids: np.ndarray):
+    """Digest selected pool blocks where they lie (the pool is only read).
+
+    Returns (status, block_digests, kv_digests, skipped).
+    """
+    pool_b = _bytes_view(pool)
+    ids = np.ascontiguousarray(ids, dtype=np.int32)
+    k = block_bytes // BLOCK
+    bd = np.zeros(len(ids) * n_planes * k, dtype=np.uint64)
+    kd = np.zeros(len(ids), dtype=np.uint64)
+    skipped = C.c_uint64(0)
+    rc = lib().gmso_kv_digest(_ptr(pool_b), plane_stride, block_stride, n_planes, n_blocks, block_bytes, _ptr(ids),
+                              len(ids), _ptr(bd), _ptr(kd), C.addressof(skipped))
     return int(rc), bd, kd, int(skipped.value)

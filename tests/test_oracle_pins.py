@@ -385,3 +385,34 @@ def test_kv_capture_is_the_inverse_of_kv_restore(oracle):
     rc2, bd2, kd2, skipped2 = oracle.kv_restore(pool2, plane_stride, bb, n_planes, n_blocks, bb, image, ips, bb, ids)
     assert rc2 == 0 and skipped2 == 2 and np.array_equal(pool2, pool)
     assert np.array_equal(bd2, bd) and np.array_equal(kd2, kd)
+
+
+def test_kv_digest_is_the_tensor_digest_of_the_block_planes_in_place(oracle):
+    rng = np.random.default_rng(53)
+    n_planes, n_blocks, bb = 4, 9, 12288
+    k = bb // 4096
+    ids = np.array([8, 0, 9, 4, -1], np.int32)  # 9 and -1 are out of range
+    plane_stride, block_stride = n_blocks * bb + 1024, bb
+    pool = rng.integers(0, 256, n_planes * plane_stride, dtype=np.uint8)
+    before = pool.copy()
+    rc, bd, kd, skipped = oracle.kv_digest(pool, plane_stride, block_stride, n_planes, n_blocks, bb, ids)
+    assert rc == 0 and skipped == 2
+    assert np.array_equal(pool, before)  # read-only
+    for j, blk in enumerate(ids):
+        ok = 0 <= blk < n_blocks
+        planes = [before[p * plane_stride + blk * block_stride :][:bb] for p in range(n_planes)] if ok else []
+        for p in range(n_planes):
+            for c in range(k):
+                want = oracle.block_digest(planes[p][c * 4096 : (c + 1) * 4096]) if ok else 0
+                assert int(bd[(j * n_planes + p) * k + c]) == want
+        assert int(kd[j]) == (oracle.tensor_digest(np.concatenate(planes))[0] if ok else 0)
+    # it is what a capture of the same blocks reports, and what restoring that capture reports
+    image = np.zeros(n_planes * len(ids) * bb, np.uint8)
+    rc, bd2, kd2, _ = oracle.kv_capture(before, plane_stride, block_stride, n_planes, n_blocks, bb, image, len(ids) * bb, bb, ids)
+    assert rc == 0 and np.array_equal(bd2, bd) and np.array_equal(kd2, kd)
+    # one flipped bit in one plane of block 4 changes exactly that 4 KiB block's digest and that slot's KV digest
+    pool[2 * plane_stride + 4 * block_stride + 5000] ^= 0x20
+    rc, bd3, kd3, _ = oracle.kv_digest(pool, plane_stride, block_stride, n_planes, n_blocks, bb, ids)
+    diff = np.nonzero(bd3 != bd)[0]
+    assert diff.tolist() == [(3 * n_planes + 2) * k + 1]
+    assert np.nonzero(kd3 != kd)[0].tolist() == [3]
