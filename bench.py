@@ -313,9 +313,11 @@ class KvBench:
         self.desc = gms.KvPool(base=self.pool.data_ptr(), plane_stride=k.plane_stride, block_stride=k.block_stride,
                                n_planes=k.n_planes, n_blocks=k.n_blocks, block_bytes=k.block_bytes)
         self.payload = k.payload_bytes
-        self.traffic = 2 * self.payload + 8 * self.bd.numel()
-        self.phase_names = ["kv_restore"]
-        self.dominant, self.dominant_bytes = "kv_restore", self.traffic
+        self.bytes_restore = 2 * self.payload + 8 * self.bd.numel()
+        self.bytes_digest = self.payload + 8 * self.bd.numel()
+        self.traffic = self.bytes_restore + self.bytes_digest
+        self.phase_names = ["kv_restore", "kv_digest"]
+        self.dominant, self.dominant_bytes = "kv_restore", self.bytes_restore
 
     def step(self, marks=None, image=None, kind=None):
         g, k = self.gms, self.k
@@ -323,6 +325,8 @@ class KvBench:
         g.gms_kv_restore(self.desc, self.image, k.img_plane_stride, k.img_slot_stride, g.SRC_DEVICE, self.ids, len(k.ids),
                          self.bd, self.kd, self.st)
         if marks: marks[1].record()
+        g.gms_kv_digest(self.desc, self.ids, len(k.ids), self.bd, self.kd, self.st)
+        if marks: marks[2].record()
 
     def check(self):
         self.torch.cuda.synchronize()
@@ -331,7 +335,7 @@ class KvBench:
     def config(self):
         k = self.k
         return {"workload": f"{k.name}: pool {k.pool_bytes} B, {len(k.ids)} of {k.n_blocks} blocks selected, {self.payload} B moved",
-                "step": "gms_kv_restore(device image)", "l2": "inputs larger than L2 (no flush)", "payload_bytes": self.payload}
+                "step": "gms_kv_restore(device image) + gms_kv_digest(the same blocks in place)", "l2": "inputs larger than L2 (no flush)", "payload_bytes": self.payload}
 
 
 def event_list(torch, n):
@@ -485,11 +489,12 @@ def cpu_baseline_kv(bench, planes=16):
     t = time.perf_counter()
     rc, bd, kd, skipped = oracle.kv_restore(pool, k.plane_stride, k.block_stride, planes, k.n_blocks, k.block_bytes, image,
                                             k.img_plane_stride, k.img_slot_stride, k.ids)
+    rc2, bd2, kd2, _ = oracle.kv_digest(pool, k.plane_stride, k.block_stride, planes, k.n_blocks, k.block_bytes, k.ids)
     dt = time.perf_counter() - t
-    assert rc == 0 and skipped == 0
+    assert rc == 0 and rc2 == 0 and skipped == 0 and (bd2 == bd).all() and (kd2 == kd).all()
     moved = planes * len(k.ids) * k.block_bytes
-    return {"value": (2 * moved + 8 * bd.size) / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"first {planes} of {k.n_planes} planes of the same pool, image and id list ({moved} B moved), "
+    return {"value": (3 * moved + 16 * bd.size) / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"kv_restore + kv_digest on the first {planes} of {k.n_planes} planes of the same pool, image and id list ({moved} B moved), "
                       f"{dt:.2f} s on 1 of {os.cpu_count()} host cores"}
 
 

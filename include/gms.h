@@ -292,6 +292,18 @@ int gms_kv_capture(const gms_kv_pool *pool, void *image, uint64_t img_plane_stri
                    uint64_t *d_kv_digests, uint64_t *d_status, void *stream);
 
 /*
+ * gms_kv_digest -- the same extension read together with Section 2.2: KV blocks that outlived an
+ * engine may be reused only if they are intact.  pool[p][d_block_ids[j]] is digested where it lies,
+ * for every plane p; nothing is written to the pool and there is no image.  Digest layout, skipping
+ * of out-of-range ids (digests 0, counted in d_status[0]) and status words are those of
+ * gms_kv_restore, so the output compares directly with what gms_kv_restore / gms_kv_capture of the
+ * same id list reported (gms_verify_flat_noalloc names the differing 4 KiB blocks).
+ * pool->flags is ignored apart from the range check.  Errors: NULL, ALIGN, ARG, RANGE, CUDA.
+ */
+int gms_kv_digest(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
+                  uint64_t *d_kv_digests, uint64_t *d_status, void *stream);
+
+/*
  * Pinned, device-mapped host memory for a GMS_SRC_HOST_MAPPED image (the
  * host-resident snapshot of Section 3.1 step 3 / Section 6).  *device_view is
  * the address to pass as `image`.

@@ -508,6 +508,7 @@ static int kv_call(const gms_kv_pool *pool, const void *image, uint64_t img_plan
     a.status = reinterpret_cast<unsigned long long *>(d_status);
     a.hints = 0;
     a.capture = capture ? 1u : 0u;
+    a.digest_only = 0u;
     a.by_id = (pool->flags & GMS_KV_IMAGE_BY_ID) ? 1u : 0u;
     GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
@@ -527,6 +528,36 @@ int gms_kv_capture(const gms_kv_pool *pool, void *image, uint64_t img_plane_stri
 {
     return kv_call(pool, image, img_plane_stride, img_slot_stride, image_kind, d_block_ids, n_sel, d_block_digests, d_kv_digests,
                    d_status, stream, true);
+}
+
+int gms_kv_digest(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
+                  uint64_t *d_kv_digests, uint64_t *d_status, void *stream)
+{
+    if (!pool || !d_status) return GMS_ERR_NULL;
+    if (pool->block_bytes == 0 || pool->block_bytes % gms::kBlockBytes) return GMS_ERR_ALIGN;
+    if (pool->block_bytes > gms::kMaxChunkBlocks * gms::kBlockBytes) return GMS_ERR_ARG;
+    const bool work = n_sel && pool->n_planes;
+    if (work && (!pool->base || !d_block_ids)) return GMS_ERR_NULL;
+    if ((reinterpret_cast<uint64_t>(pool->base) | pool->plane_stride | pool->block_stride) & 15u) return GMS_ERR_ALIGN;
+    if (pool->block_stride < pool->block_bytes && pool->n_blocks > 1) return GMS_ERR_ARG;
+    if (pool->flags & ~GMS_KV_IMAGE_BY_ID) return GMS_ERR_ARG;
+    const uint64_t k = pool->block_bytes / gms::kBlockBytes;
+    if ((uint64_t)n_sel * pool->n_planes * k >= 0xffffffffull) return GMS_ERR_RANGE;
+    gms::KvArgs a = {};
+    a.pool_base = static_cast<uint8_t *>(pool->base);
+    a.plane_stride = pool->plane_stride;
+    a.block_stride = pool->block_stride;
+    a.n_planes = pool->n_planes;
+    a.n_blocks = pool->n_blocks;
+    a.block_bytes = pool->block_bytes;
+    a.ids = d_block_ids;
+    a.n_sel = n_sel;
+    a.block_digests = d_block_digests;
+    a.kv_digests = d_kv_digests;
+    a.status = reinterpret_cast<unsigned long long *>(d_status);
+    a.digest_only = 1u;
+    GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
+    return GMS_OK;
 }
 
 int gms_host_image_alloc(uint64_t nbytes, void **host_ptr, void **device_view)

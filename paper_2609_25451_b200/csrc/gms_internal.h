@@ -39,7 +39,7 @@ struct Geometry {
     uint32_t counters; // work counters the chunk claims are spread over
     uint32_t group;    // consecutive chunks bought by one claim
 };
-enum Kind { kRestore = 0, kDigest = 1, kKv = 2 };  // the three streaming kernels have their own shapes
+enum Kind { kRestore = 0, kDigest = 1, kKv = 2, kKvDigest = 3, kKinds = 4 };  // each streaming kernel has its own shape
 cudaError_t get_geometry(Kind kind, Geometry *g);
 
 struct StreamArgs {
@@ -71,7 +71,8 @@ struct KvArgs {
     uint64_t *kv_digests;          // may be null
     unsigned long long *status;    // [0] skipped ids, [1] device status word, [2] work counter, [3] spare
     uint32_t capture;              // 1: gather pool blocks into the image
-    uint32_t by_id;                // 1: the image is pool-shaped (slot = block id), else packed (slot = list position)
+    uint32_t digest_only;          // 1: digest the selected pool blocks where they lie (no image, nothing written)
+    uint32_t by_id;               // 1: the image is pool-shaped (slot = block id), else packed (slot = list position)
     uint32_t hints;                // filled in by the launcher
 };
 

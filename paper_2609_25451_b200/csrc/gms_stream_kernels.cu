@@ -316,8 +316,8 @@ struct KvProvider {
             const uint32_t img_slot = a.by_id ? (uint32_t)id : j;  // pool-shaped image: slot = block id
             uint8_t *img = const_cast<uint8_t *>(a.image) + (uint64_t)p * a.img_plane_stride + (uint64_t)img_slot * a.img_slot_stride;
             uint8_t *blk = a.pool_base + (uint64_t)p * a.plane_stride + (uint64_t)id * a.block_stride;
-            it.src = a.capture ? blk : img;
-            it.dst = a.capture ? img : blk;
+            it.src = (a.capture || a.digest_only) ? blk : img;
+            it.dst = a.capture ? img : blk;  // unused when digesting in place
             it.nbytes = a.block_bytes;
             it.tensor = j;
             it.gblock0 = slot0;
@@ -532,7 +532,7 @@ __global__ void __launch_bounds__(512, 1) gms_stream_kernel(StreamArgs a)
     run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.hints);
 }
 
-template <int S>
+template <int S, bool kStore>
 __global__ void __launch_bounds__(512, 1) gms_kv_stream_kernel(KvArgs a)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -543,7 +543,7 @@ __global__ void __launch_bounds__(512, 1) gms_kv_stream_kernel(KvArgs a)
     prov.total = a.n_sel * a.n_planes;
     asm volatile("griddepcontrol.wait;" ::: "memory");
     prov.init(threadIdx.x & 31u);
-    run_pipeline<S, true>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, a.hints);
+    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, a.hints);
 }
 
 // Clears the accumulators the streaming kernels XOR / add into.
@@ -577,13 +577,14 @@ cudaError_t set_attrs(Kind kind, uint32_t smem)
 {
     const void *f = kind == kRestore ? (const void *)gms_stream_kernel<S, true>
                     : kind == kDigest ? (const void *)gms_stream_kernel<S, false>
-                                      : (const void *)gms_kv_stream_kernel<S>;
+                    : kind == kKv     ? (const void *)gms_kv_stream_kernel<S, true>
+                                      : (const void *)gms_kv_stream_kernel<S, false>;
     return cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
 constexpr int kMaxDevices = 64;
-Geometry g_geom[kMaxDevices][3];
-bool g_geom_ok[kMaxDevices][3];
+Geometry g_geom[kMaxDevices][kKinds];
+bool g_geom_ok[kMaxDevices][kKinds];
 
 cudaError_t prologue(uint64_t *accum, uint64_t n_accum, unsigned int *counters, uint32_t n_counters, unsigned long long *status,
                      uint32_t n_status, cudaStream_t s)
@@ -660,7 +661,7 @@ cudaError_t get_geometry(Kind kind, Geometry *out)
         Geometry g;
         uint32_t per_sm = 1;
         // defaults are what the benchmark numbers were taken with
-        if (kind == kDigest) {
+        if (kind == kDigest || kind == kKvDigest) {
             g.warps = 16, g.stages = 3;
             env_geom("GMS_GEOM_DIGEST", g.warps, g.stages, per_sm);
         } else if (kind == kRestore) {
@@ -705,17 +706,26 @@ cudaError_t launch_digest(const StreamArgs &a, cudaStream_t s) { return launch_s
 cudaError_t launch_kv_restore(const KvArgs &a, cudaStream_t s)
 {
     Geometry g;
-    cudaError_t e = get_geometry(kKv, &g);
+    cudaError_t e = get_geometry(a.digest_only ? kKvDigest : kKv, &g);
     if (e) return e;
     if ((e = prologue(a.kv_digests, a.n_sel, nullptr, 0, a.status, 4, s))) return e;
     if (a.n_sel == 0 || a.n_planes == 0) return cudaSuccess;
     KvArgs b = a;
     b.hints = g.hints;
-    switch (g.stages) {
-    case 3: e = launch_after_prologue(gms_kv_stream_kernel<3>, g, s, b); break;
-    case 6: e = launch_after_prologue(gms_kv_stream_kernel<6>, g, s, b); break;
-    case 8: e = launch_after_prologue(gms_kv_stream_kernel<8>, g, s, b); break;
-    default: e = launch_after_prologue(gms_kv_stream_kernel<4>, g, s, b); break;
+    if (a.digest_only) {
+        switch (g.stages) {
+        case 3: e = launch_after_prologue(gms_kv_stream_kernel<3, false>, g, s, b); break;
+        case 6: e = launch_after_prologue(gms_kv_stream_kernel<6, false>, g, s, b); break;
+        case 8: e = launch_after_prologue(gms_kv_stream_kernel<8, false>, g, s, b); break;
+        default: e = launch_after_prologue(gms_kv_stream_kernel<4, false>, g, s, b); break;
+        }
+    } else {
+        switch (g.stages) {
+        case 3: e = launch_after_prologue(gms_kv_stream_kernel<3, true>, g, s, b); break;
+        case 6: e = launch_after_prologue(gms_kv_stream_kernel<6, true>, g, s, b); break;
+        case 8: e = launch_after_prologue(gms_kv_stream_kernel<8, true>, g, s, b); break;
+        default: e = launch_after_prologue(gms_kv_stream_kernel<4, true>, g, s, b); break;
+        }
     }
     count_launches(1);
     return e;

@@ -33,7 +33,7 @@ MISMATCH_DTYPE = np.dtype([("tensor_id", "<u8"), ("block", "<u8")])
 EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
-    "gms_verify", "gms_verify_tensors", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_host_image_alloc", "gms_host_image_free",
+    "gms_verify", "gms_verify_tensors", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_kv_digest", "gms_host_image_alloc", "gms_host_image_free",
     "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd", "gms_stage_create", "gms_stage_destroy", "gms_restore_staged",
     "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
     "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
@@ -88,6 +88,7 @@ def lib():
             "gms_last_device_status": (i, [p, p, pu64]),
             "gms_kv_restore": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
             "gms_kv_capture": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
+            "gms_kv_digest": (i, [C.POINTER(KvPool), p, u32, p, p, p, p]),
             "gms_host_image_alloc": (i, [u64, pp, pp]),
             "gms_host_image_free": (i, [p]),
             "gms_pipe_create": (i, [u32, u64, u32, pp]),
@@ -246,6 +247,11 @@ def gms_kv_capture(pool: KvPool, image, img_plane_stride: int, img_slot_stride: 
     _check(lib().gms_kv_capture(C.byref(pool), _dev(image), img_plane_stride, img_slot_stride, image_kind,
                                 _dev(d_block_ids), n_sel, _dev(d_block_digests), _dev(d_kv_digests), _dev(d_status),
                                 _stream(stream)), "gms_kv_capture")
+
+
+def gms_kv_digest(pool: KvPool, d_block_ids, n_sel: int, d_block_digests, d_kv_digests, d_status, stream=None):
+    _check(lib().gms_kv_digest(C.byref(pool), _dev(d_block_ids), n_sel, _dev(d_block_digests), _dev(d_kv_digests),
+                               _dev(d_status), _stream(stream)), "gms_kv_digest")
 
 
 def gms_host_image_alloc(nbytes: int):

@@ -234,6 +234,13 @@ def test_kv_pool_full_size(oracle):
         planes = img3[:, j, :].cpu().numpy()
         T, obd = oracle.tensor_digest(planes.reshape(-1))
         assert int(kd_h[j]) == T and np.array_equal(bd_h[j].reshape(-1), obd), j
+    # digesting the same blocks where they now lie gives the same digests and writes nothing
+    bd2, kd2 = torch.zeros_like(bd), torch.zeros_like(kd)
+    gms.gms_kv_digest(desc, ids, n_sel, bd2, kd2, st)
+    torch.cuda.synchronize()
+    assert st[:2].tolist() == [0, 0]
+    assert torch.equal(bd2, bd) and torch.equal(kd2, kd)
+    assert torch.equal(pool.view(torch.int64).view(k.n_planes * k.n_blocks, -1).sum(dim=1), sums_after)
 
 
 def test_host_sourced_70b_shard_full_size(oracle):
