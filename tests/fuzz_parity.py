@@ -23,7 +23,7 @@ from oracle import gms_oracle as oracle  # noqa: E402
 from paper_2609_25451_b200 import gms  # noqa: E402
 from paper_2609_25451_b200 import workloads as W  # noqa: E402
 
-from gpu_harness import FILL, DeviceWorkload, guarded_u64, oracle_record, payload_of, PAD  # noqa: E402
+from gpu_harness import CANARY, FILL, DeviceWorkload, guarded_u64, oracle_record, payload_of, PAD  # noqa: E402
 
 
 def random_sizes(rng):
@@ -132,6 +132,17 @@ def one_kv_round(rng):
     assert int(status[0]) == oskip and int(status[1]) == 0, "kv status differs"
     assert np.array_equal(pool.cpu().numpy(), want_pool) and np.array_equal(img.cpu().numpy(), want_img), "kv bytes differ"
     assert np.array_equal(payload_of(bd, n_sel * n_planes * k), obd) and np.array_equal(payload_of(kd, n_sel), okd), "kv digests"
+    # the selected blocks digested where they now lie, against the oracle's in-place digest of the expected pool
+    rc, obd2, okd2, oskip2 = oracle.kv_digest(want_pool, plane_stride, bb, n_planes, n_blocks, bb, ids)
+    assert rc == 0
+    bd.fill_(CANARY)
+    kd.fill_(CANARY)
+    gms.gms_kv_digest(desc, ids_d, n_sel, bd.data_ptr() + 8 * PAD, kd.data_ptr() + 8 * PAD, st.data_ptr() + 8 * PAD)
+    torch.cuda.synchronize()
+    status = payload_of(st, 4)
+    assert int(status[0]) == oskip2 and int(status[1]) == 0, "kv digest status differs"
+    assert np.array_equal(pool.cpu().numpy(), want_pool), "kv digest wrote to the pool"
+    assert np.array_equal(payload_of(bd, n_sel * n_planes * k), obd2) and np.array_equal(payload_of(kd, n_sel), okd2), "kv in-place digests"
 
 
 def main():
