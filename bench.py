@@ -16,9 +16,10 @@ bf16 bit patterns); image and destinations are resident in HBM when the timed re
 `value` is algorithmic HBM traffic per second over the whole step (bytes the method must read and
 write: payload once for the digest pass, twice for the restore pass, plus 8 B per 4 KiB of digests
 and the verify pass's 16 B per block), summed over all GPUs, timed on the device with CUDA events,
-max over ranks.  `e2e` is the same metric with the snapshot image in pinned host memory: the
-restore kernel pulls it across the host link inside the timed region and the verdict (mismatch
-count, tensor digests) is read back to the host every step.  With N > 1 every rank restores its own
+max over ranks.  `e2e` is the same metric with the snapshot image in pinned host memory:
+gms_restore_staged moves it across the host link inside the timed region (copy engine -> device
+ring -> restore kernel) and the verdict (mismatch count, tensor digests) is read back to the host
+every step.  With N > 1 every rank restores its own
 replica (the path has no exchange step): weak scaling, no data-path collective.
 """
 from __future__ import annotations
