@@ -1,8 +1,8 @@
 // gms_restore_fd: storage -> pinned host buffers -> device allocations, pipelined.
 //
-// Section 4 (GMS paragraph) has a read-write client repopulate a cold service "from storage in
-// parallel with process restoration"; Section 3.1 prices that at S / B_eff and Section 3.3 notes that
-// runtime-state restoration leaves storage bandwidth unused.  This file is that leg: the snapshot
+// Section 4 (GMS paragraph) has a fresh writer fill a cold service from storage while the process
+// itself is being restored; Section 3.1 prices that at S / B_eff and Section 3.3 notes that restoring
+// the runtime state leaves storage bandwidth unused.  This file is that leg: the snapshot
 // image is never resident as a whole.  A small ring of pinned, device-mapped buffers is filled by a
 // pool of reader threads (pread), and as soon as a buffer holds a window of the image the restore
 // kernel is launched on the chunks whose sources lie in that window, reading the pinned buffer
