@@ -1,10 +1,10 @@
 // gms_service_*: the substrate under the destinations -- service-owned device allocations with the
 // paper's ownership protocol, in one process.
 //
-// Section 4 (GMS paragraph): the service creates physical allocations with cuMemCreate; "to
-// amortize VMM operations, the pool uses a first-fit suballocator over 2 GiB slabs, with larger
-// dedicated slabs for individual allocations exceeding 2 GiB", so mapping and permission set-up
-// happen per slab, not per tensor.  Section 3.2 / Figure (ownership protocol): EMPTY -> RW (one
+// Section 4 (GMS paragraph): the service creates physical allocations with cuMemCreate and keeps
+// the number of VMM calls down by suballocating, first fit, out of 2 GiB slabs, giving any single
+// allocation above 2 GiB a slab of its own, so mapping and permission set-up happen per slab, not
+// per tensor.  Section 3.2 / Figure (ownership protocol): EMPTY -> RW (one
 // writer populates) -> COMMITTED (immutable, no readers) <-> RO (n >= 1 readers); a writer that
 // gives up before commit discards the state; write access is available again once the last
 // reader has left; read-only access is enforced with cuMemSetAccess.
