@@ -87,6 +87,31 @@ def test_random_invalid_records_agree_with_oracle(oracle):
     assert agree > 150
 
 
+def test_index_limits_are_refused_before_anything_is_built():
+    # digest slots are 32-bit on the device: 2^32 - 1 blocks or more (16 TiB of payload) is refused during validation
+    big = 4096 * (2**32 - 1)
+    ent = gms.make_entries([(1, 0, FAKE_BASE, big)])
+    with pytest.raises(gms.GmsError) as ei:
+        gms.gms_manifest_build(ent, big, gms.BUILD_HOST_ONLY)
+    assert ei.value.status == gms.ERR_RANGE
+    # the same limit reached by the sum over two tensors
+    half = 4096 * 2**31
+    ent = gms.make_entries([(1, 0, FAKE_BASE, half), (2, half, FAKE_BASE + half, half)])
+    with pytest.raises(gms.GmsError) as ei:
+        gms.gms_manifest_build(ent, 2 * half, gms.BUILD_HOST_ONLY)
+    assert ei.value.status == gms.ERR_RANGE
+    # a destination range that wraps the address space
+    ent = gms.make_entries([(1, 0, 2**64 - 4096, 8192)])
+    with pytest.raises(gms.GmsError) as ei:
+        gms.gms_manifest_build(ent, 8192, gms.BUILD_HOST_ONLY)
+    assert ei.value.status == gms.ERR_RANGE
+    # a byte range of 100 GB in one tensor is fine on the host (25 M blocks, 6 M chunks)
+    n = 100 * 10**9
+    m = gms.gms_manifest_build(gms.make_entries([(1, 0, FAKE_BASE, n)]), n, gms.BUILD_HOST_ONLY)
+    assert m.n_blocks == (n + 4095) // 4096 and gms.gms_manifest_chunk_count(m) == (m.n_blocks + 3) // 4
+    m.close()
+
+
 def test_null_and_flag_errors():
     out = ctypes.c_void_p()
     assert gms.lib().gms_manifest_build(None, 3, 100, 0, ctypes.byref(out)) == gms.ERR_NULL
