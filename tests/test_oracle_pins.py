@@ -416,3 +416,17 @@ def test_kv_digest_is_the_tensor_digest_of_the_block_planes_in_place(oracle):
     diff = np.nonzero(bd3 != bd)[0]
     assert diff.tolist() == [(3 * n_planes + 2) * k + 1]
     assert np.nonzero(kd3 != kd)[0].tolist() == [3]
+
+
+def test_oracle_has_not_drifted_from_its_stored_outputs(oracle):
+    """tests/golden/oracle_regression.txt was written by tests/golden/make_oracle_regression.py, which calls only the
+    oracle: a drift alarm (any later change to the oracle's arithmetic must be deliberate), not a correctness pin."""
+    import importlib.util
+    import os
+
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_oracle_regression", os.path.join(here, "make_oracle_regression.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    with open(os.path.join(here, "oracle_regression.txt")) as f:
+        assert f.read() == mod.render()
