@@ -316,27 +316,37 @@ class KvBench:
         self.payload = k.payload_bytes
         self.bytes_restore = 2 * self.payload + 8 * self.bd.numel()
         self.bytes_digest = self.payload + 8 * self.bd.numel()
-        self.traffic = self.bytes_restore + self.bytes_digest
-        self.phase_names = ["kv_restore", "kv_digest"]
+        self.bytes_verify = 16 * self.bd.numel()
+        self.traffic = self.bytes_restore + self.bytes_digest + self.bytes_verify
+        self.phase_names = ["kv_restore", "kv_digest", "kv_verify"]
         self.dominant, self.dominant_bytes = "kv_restore", self.bytes_restore
+        # digests of the restore, against which the in-place digests are verified (allocation-free flat verify)
+        self.bd_restore = torch.zeros_like(self.bd)
+        self.mm = torch.zeros(2 * 64, dtype=torch.int64, device=dev)
+        self.cnt = torch.zeros(1, dtype=torch.int64, device=dev)
+        self.flat_verify = self.bd.numel() <= 4194304  # the entry point's fixed scratch
 
     def step(self, marks=None, image=None, kind=None):
         g, k = self.gms, self.k
         if marks: marks[0].record()
         g.gms_kv_restore(self.desc, self.image, k.img_plane_stride, k.img_slot_stride, g.SRC_DEVICE, self.ids, len(k.ids),
-                         self.bd, self.kd, self.st)
+                         self.bd_restore, self.kd, self.st)
         if marks: marks[1].record()
         g.gms_kv_digest(self.desc, self.ids, len(k.ids), self.bd, self.kd, self.st)
         if marks: marks[2].record()
+        if self.flat_verify:
+            g.gms_verify_flat_noalloc(self.bd, self.bd_restore, self.bd.numel(), 0, self.mm, 64, self.cnt)
+        if marks: marks[3].record()
 
     def check(self):
         self.torch.cuda.synchronize()
         assert self.st[:2].tolist() == [0, 0]
+        assert int(self.cnt.item()) == 0, "in-place KV digests differ from the ones the restore reported"
 
     def config(self):
         k = self.k
         return {"workload": f"{k.name}: pool {k.pool_bytes} B, {len(k.ids)} of {k.n_blocks} blocks selected, {self.payload} B moved",
-                "step": "gms_kv_restore(device image) + gms_kv_digest(the same blocks in place)", "l2": "inputs larger than L2 (no flush)", "payload_bytes": self.payload}
+                "step": "gms_kv_restore(device image) + gms_kv_digest(the same blocks in place) + gms_verify_flat_noalloc", "l2": "inputs larger than L2 (no flush)", "payload_bytes": self.payload}
 
 
 def event_list(torch, n):
