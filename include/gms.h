@@ -390,6 +390,8 @@ typedef struct {
     uint64_t slab_bytes;           /* regular slab size after rounding to the mapping granularity */
     uint64_t bytes_reserved;       /* sum of slab sizes                                           */
     uint64_t bytes_allocated;      /* sum of (256-byte rounded) allocation sizes                  */
+    uint32_t attached;             /* 0 between gms_service_detach and gms_service_reattach        */
+    uint32_t backed;               /* 0 between gms_service_release_pages and gms_service_back_pages */
 } gms_service_stats;
 int gms_service_create(uint64_t slab_bytes, uint32_t flags, gms_service **out);
 int gms_service_destroy(gms_service *s);
@@ -401,6 +403,29 @@ int gms_service_acquire_ro(gms_service *s);
 int gms_service_release_ro(gms_service *s);
 int gms_service_info(gms_service *s, gms_service_stats *out);
 int gms_service_access(gms_service *s, const void *dptr, uint32_t *writable);
+
+/*
+ * Addresses that outlive their mappings.  A snapshot of an engine holds the virtual addresses of its
+ * tensors (in CUDA graphs and tensor metadata) but none of the memory behind them, so both calls
+ * below keep every virtual range reserved: the destination pointers of a manifest built before
+ * stay valid afterwards.
+ *   detach / reattach           Section 3.3: before capture the engine unmaps each service range but
+ *       keeps its address reservation while the service keeps the physical memory; after restore the
+ *       surviving memory is mapped read-only at the same addresses.  COMMITTED (no readers) only.
+ *       Between the two calls nothing may touch the addresses (gms_service_access returns
+ *       GMS_ERR_STATE) and acquire_rw / acquire_ro are refused.  Contents are preserved.
+ *   release_pages / back_pages  Section 3.1 (pages released before capture, fresh pages mapped at the
+ *       same addresses after restore) and Section 3.3 (after a device-invalidating failure the state
+ *       is rebuilt in fresh allocations): RW only.  The physical memory of every slab is given back
+ *       to the driver; back_pages maps fresh memory, writable, whose contents are undefined until the
+ *       writer restores them (gms_restore, gms_kv_restore).  In between, alloc / commit are refused.
+ * Both pairs synchronise the device first.  Errors: NULL, STATE, NOMEM (back_pages; the service then
+ * stays without pages), CUDA.
+ */
+int gms_service_detach(gms_service *s);
+int gms_service_reattach(gms_service *s);
+int gms_service_release_pages(gms_service *s);
+int gms_service_back_pages(gms_service *s);
 
 /* Launch geometry of the streaming kernels on the current device (for reporting). */
 int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *smem_bytes);

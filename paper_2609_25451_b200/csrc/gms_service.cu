@@ -91,6 +91,8 @@ struct gms_service {
     uint64_t slab_bytes = 0, granularity = 2ull << 20;
     uint64_t fake_next_va = 0x700000000000ull;
     uint32_t state = GMS_STATE_EMPTY, readers = 0;
+    bool attached = true;  // slabs are mapped into the address space (false between detach and reattach)
+    bool backed = true;    // slabs have physical memory (false between release_pages and back_pages)
     std::vector<Slab> slabs;
 };
 
@@ -149,11 +151,19 @@ void drop_slab(gms_service *s, Slab &slab)
 {
     if (!s->dry_run && slab.va) {
         Driver *d = driver();
-        d->memUnmap((CUdeviceptr)slab.va, slab.size);
+        if (s->attached && s->backed) d->memUnmap((CUdeviceptr)slab.va, slab.size);
         d->memAddressFree((CUdeviceptr)slab.va, slab.size);
-        d->memRelease(slab.handle);
+        if (s->backed) d->memRelease(slab.handle);
     }
     slab.va = 0;
+}
+
+// Maps the slab's physical memory at its reserved address again, with the given access.
+int map_slab(gms_service *s, Slab &slab, bool writable)
+{
+    if (s->dry_run) return GMS_OK;
+    if (driver()->memMap((CUdeviceptr)slab.va, slab.size, 0, slab.handle, 0) != CUDA_SUCCESS) return GMS_ERR_CUDA;
+    return set_access(s, slab, writable);
 }
 
 // first fit inside one slab
@@ -243,7 +253,7 @@ int gms_service_acquire_rw(gms_service *s)
         s->state = GMS_STATE_RW;
         return GMS_OK;
     }
-    if (s->state != GMS_STATE_COMMITTED) return GMS_ERR_STATE;  // a writer or readers hold it
+    if (s->state != GMS_STATE_COMMITTED || !s->attached) return GMS_ERR_STATE;  // a writer or readers hold it, or it is detached
     int rc = quiesce(s);
     for (Slab &slab : s->slabs)
         if (rc == GMS_OK) rc = set_access(s, slab, true);
@@ -257,7 +267,7 @@ int gms_service_alloc(gms_service *s, uint64_t nbytes, void **dptr)
     if (!s || !dptr) return GMS_ERR_NULL;
     *dptr = nullptr;
     std::lock_guard<std::mutex> l(s->mu);
-    if (s->state != GMS_STATE_RW) return GMS_ERR_STATE;
+    if (s->state != GMS_STATE_RW || !s->backed) return GMS_ERR_STATE;
     if (nbytes == 0 || nbytes > (1ull << 46)) return GMS_ERR_ARG;
     const uint64_t need = (nbytes + kAllocAlign - 1) / kAllocAlign * kAllocAlign;
     uint64_t off = 0;
@@ -288,7 +298,7 @@ int gms_service_commit(gms_service *s)
 {
     if (!s) return GMS_ERR_NULL;
     std::lock_guard<std::mutex> l(s->mu);
-    if (s->state != GMS_STATE_RW) return GMS_ERR_STATE;
+    if (s->state != GMS_STATE_RW || !s->backed) return GMS_ERR_STATE;
     int rc = quiesce(s);
     for (Slab &slab : s->slabs)
         if (rc == GMS_OK) rc = set_access(s, slab, false);
@@ -305,14 +315,100 @@ int gms_service_abort(gms_service *s)
     int rc = quiesce(s);
     discard_all(s);
     s->state = GMS_STATE_EMPTY;
+    s->backed = true;
     return rc;
+}
+
+int gms_service_detach(gms_service *s)
+{
+    if (!s) return GMS_ERR_NULL;
+    std::lock_guard<std::mutex> l(s->mu);
+    if (s->state != GMS_STATE_COMMITTED || !s->attached) return GMS_ERR_STATE;
+    int rc = quiesce(s);
+    if (rc != GMS_OK) return rc;
+    if (!s->dry_run)
+        for (Slab &slab : s->slabs)
+            if (driver()->memUnmap((CUdeviceptr)slab.va, slab.size) != CUDA_SUCCESS) rc = GMS_ERR_CUDA;
+    s->attached = false;
+    return rc;
+}
+
+int gms_service_reattach(gms_service *s)
+{
+    if (!s) return GMS_ERR_NULL;
+    std::lock_guard<std::mutex> l(s->mu);
+    if (s->state != GMS_STATE_COMMITTED || s->attached) return GMS_ERR_STATE;
+    int rc = GMS_OK;
+    for (Slab &slab : s->slabs)
+        if (rc == GMS_OK) rc = map_slab(s, slab, false);  // committed state comes back read-only, at the same addresses
+    if (rc != GMS_OK) return rc;
+    s->attached = true;
+    return GMS_OK;
+}
+
+int gms_service_release_pages(gms_service *s)
+{
+    if (!s) return GMS_ERR_NULL;
+    std::lock_guard<std::mutex> l(s->mu);
+    if (s->state != GMS_STATE_RW || !s->backed) return GMS_ERR_STATE;
+    int rc = quiesce(s);
+    if (rc != GMS_OK) return rc;
+    if (!s->dry_run)
+        for (Slab &slab : s->slabs) {
+            if (driver()->memUnmap((CUdeviceptr)slab.va, slab.size) != CUDA_SUCCESS) rc = GMS_ERR_CUDA;
+            if (driver()->memRelease(slab.handle) != CUDA_SUCCESS) rc = GMS_ERR_CUDA;
+            slab.handle = 0;
+        }
+    s->backed = false;
+    return rc;
+}
+
+int gms_service_back_pages(gms_service *s)
+{
+    if (!s) return GMS_ERR_NULL;
+    std::lock_guard<std::mutex> l(s->mu);
+    if (s->state != GMS_STATE_RW || s->backed) return GMS_ERR_STATE;
+    if (!s->dry_run) {
+        Driver *d = driver();
+        CUmemAllocationProp prop = {};
+        prop.type = CU_MEM_ALLOCATION_TYPE_PINNED;
+        prop.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
+        prop.location.id = s->device;
+        size_t done = 0;
+        int rc = GMS_OK;
+        for (; done < s->slabs.size() && rc == GMS_OK; ++done) {
+            Slab &slab = s->slabs[done];
+            const CUresult r = d->memCreate(&slab.handle, slab.size, &prop, 0);
+            if (r != CUDA_SUCCESS) {
+                rc = r == CUDA_ERROR_OUT_OF_MEMORY ? GMS_ERR_NOMEM : GMS_ERR_CUDA;
+                break;
+            }
+            rc = map_slab(s, slab, true);
+            if (rc != GMS_OK) {
+                (void)d->memUnmap((CUdeviceptr)slab.va, slab.size);  // in case the mapping was made and only the access failed
+                d->memRelease(slab.handle);
+                slab.handle = 0;
+                break;
+            }
+        }
+        if (rc != GMS_OK) {  // undo: the service stays without pages, every address still reserved
+            for (size_t i = 0; i < done; ++i) {
+                d->memUnmap((CUdeviceptr)s->slabs[i].va, s->slabs[i].size);
+                d->memRelease(s->slabs[i].handle);
+                s->slabs[i].handle = 0;
+            }
+            return rc;
+        }
+    }
+    s->backed = true;
+    return GMS_OK;
 }
 
 int gms_service_acquire_ro(gms_service *s)
 {
     if (!s) return GMS_ERR_NULL;
     std::lock_guard<std::mutex> l(s->mu);
-    if (s->state != GMS_STATE_COMMITTED && s->state != GMS_STATE_RO) return GMS_ERR_STATE;
+    if ((s->state != GMS_STATE_COMMITTED && s->state != GMS_STATE_RO) || !s->attached) return GMS_ERR_STATE;
     s->state = GMS_STATE_RO;
     ++s->readers;
     return GMS_OK;
@@ -336,6 +432,8 @@ int gms_service_info(gms_service *s, gms_service_stats *out)
     st.readers = s->readers;
     st.n_slabs = s->slabs.size();
     st.slab_bytes = s->slab_bytes;
+    st.attached = s->attached ? 1u : 0u;
+    st.backed = s->backed ? 1u : 0u;
     for (const Slab &slab : s->slabs) {
         st.bytes_reserved += slab.size;
         st.bytes_allocated += slab.used;
@@ -352,6 +450,7 @@ int gms_service_access(gms_service *s, const void *dptr, uint32_t *writable)
     const uint64_t p = reinterpret_cast<uint64_t>(dptr);
     for (const Slab &slab : s->slabs) {
         if (p < slab.va || p >= slab.va + slab.size) continue;
+        if (!s->attached || !s->backed) return GMS_ERR_STATE;  // the address is reserved but nothing is mapped there
         if (s->dry_run) {
             *writable = s->state == GMS_STATE_RW ? 1u : 0u;
             return GMS_OK;

@@ -37,6 +37,7 @@ EXPORTS = (
     "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd", "gms_stage_create", "gms_stage_destroy", "gms_restore_staged",
     "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
     "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
+    "gms_service_detach", "gms_service_reattach", "gms_service_release_pages", "gms_service_back_pages",
     "gms_launch_geometry", "gms_kernel_launches", "gms_set_device", "gms_strerror", "gms_last_cuda_error", "gms_version",
 )
 
@@ -107,6 +108,10 @@ def lib():
             "gms_service_release_ro": (i, [p]),
             "gms_service_info": (i, [p, p]),
             "gms_service_access": (i, [p, p, pu32]),
+            "gms_service_detach": (i, [p]),
+            "gms_service_reattach": (i, [p]),
+            "gms_service_release_pages": (i, [p]),
+            "gms_service_back_pages": (i, [p]),
             "gms_launch_geometry": (i, [pu32, pu32, pu32]),
             "gms_kernel_launches": (u64, []),
             "gms_set_device": (i, [i]),
@@ -330,7 +335,8 @@ SERVICE_DRY_RUN = 1
 
 class ServiceStats(C.Structure):
     _fields_ = [("state", C.c_uint32), ("readers", C.c_uint32), ("n_slabs", C.c_uint64), ("n_dedicated", C.c_uint64),
-                ("slab_bytes", C.c_uint64), ("bytes_reserved", C.c_uint64), ("bytes_allocated", C.c_uint64)]
+                ("slab_bytes", C.c_uint64), ("bytes_reserved", C.c_uint64), ("bytes_allocated", C.c_uint64),
+                ("attached", C.c_uint32), ("backed", C.c_uint32)]
 
 
 class Service:
@@ -390,6 +396,22 @@ def gms_service_access(s: Service, dptr: int) -> bool:
     w = C.c_uint32()
     _check(lib().gms_service_access(s.handle, int(dptr), C.byref(w)), "gms_service_access")
     return bool(w.value)
+
+
+def gms_service_detach(s: Service):
+    _check(lib().gms_service_detach(s.handle), "gms_service_detach")
+
+
+def gms_service_reattach(s: Service):
+    _check(lib().gms_service_reattach(s.handle), "gms_service_reattach")
+
+
+def gms_service_release_pages(s: Service):
+    _check(lib().gms_service_release_pages(s.handle), "gms_service_release_pages")
+
+
+def gms_service_back_pages(s: Service):
+    _check(lib().gms_service_back_pages(s.handle), "gms_service_back_pages")
 
 
 def gms_launch_geometry():

@@ -178,3 +178,111 @@ def test_oversized_allocation_gets_a_dedicated_slab():
     assert torch.equal(back[:n], image[:n])
     m.close()
     svc.close()
+
+
+def test_detach_and_page_release_transitions_dry_run():
+    s = gms.gms_service_create(8 * MiB, gms.SERVICE_DRY_RUN)
+    info = lambda: gms.gms_service_info(s)
+    assert info()["attached"] == 1 and info()["backed"] == 1
+    # nothing to detach or release before there is state
+    for fn in (gms.gms_service_detach, gms.gms_service_reattach, gms.gms_service_release_pages, gms.gms_service_back_pages):
+        assert status_of(fn, s) == gms.ERR_STATE
+    gms.gms_service_acquire_rw(s)
+    p = gms.gms_service_alloc(s, 5000)
+    # RW: pages may be released and brought back; the books and the addresses stay
+    assert status_of(gms.gms_service_detach, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_back_pages, s) == gms.ERR_STATE
+    gms.gms_service_release_pages(s)
+    assert info()["backed"] == 0 and info()["bytes_allocated"] == 5120 and info()["n_slabs"] == 1
+    assert status_of(gms.gms_service_release_pages, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_alloc, s, 10) == gms.ERR_STATE
+    assert status_of(gms.gms_service_commit, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_access, s, p) == gms.ERR_STATE
+    gms.gms_service_back_pages(s)
+    assert info()["backed"] == 1 and gms.gms_service_access(s, p) is True
+    q = gms.gms_service_alloc(s, 10)
+    assert q != p
+    gms.gms_service_commit(s)
+    # COMMITTED: detach / reattach; no lease can be taken in between
+    assert status_of(gms.gms_service_release_pages, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_reattach, s) == gms.ERR_STATE
+    gms.gms_service_detach(s)
+    assert info()["attached"] == 0 and info()["state"] == gms.STATE_COMMITTED
+    assert status_of(gms.gms_service_detach, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_acquire_ro, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_acquire_rw, s) == gms.ERR_STATE
+    assert status_of(gms.gms_service_access, s, p) == gms.ERR_STATE
+    gms.gms_service_reattach(s)
+    assert info()["attached"] == 1 and gms.gms_service_access(s, p) is False
+    gms.gms_service_acquire_ro(s)
+    assert status_of(gms.gms_service_detach, s) == gms.ERR_STATE  # a reader holds it
+    gms.gms_service_release_ro(s)
+    # a writer that gives up while the pages are released leaves a clean, empty service
+    gms.gms_service_acquire_rw(s)
+    gms.gms_service_release_pages(s)
+    gms.gms_service_abort(s)
+    assert info()["state"] == gms.STATE_EMPTY and info()["backed"] == 1 and info()["n_slabs"] == 0
+    s.close()
+
+
+@pytest.mark.gpu
+def test_addresses_outlive_their_mappings(oracle):
+    """A manifest built once stays valid across detach / reattach (contents preserved, read-only) and across
+    release_pages / back_pages (fresh memory at the same addresses, refilled by gms_restore)."""
+    import torch
+
+    from gpu_harness import oracle_record
+
+    w = W.mixed_manifest(n_small=300, n_large=2, large_bytes=(5 * MiB) + 24, round16=False, seed=211)
+    image_h = W.random_bytes_host(w.image_bytes, seed=212)
+    svc = gms.gms_service_create(8 * MiB)
+    gms.gms_service_acquire_rw(svc)
+    ptrs = [gms.gms_service_alloc(svc, max(1, int(r["nbytes"]))) for r in w.rows]
+    image = torch.from_numpy(image_h).cuda()
+    m = gms.gms_manifest_build(gms.make_entries((r["tensor_id"], r["src_offset"], p, r["nbytes"]) for r, p in zip(w.rows, ptrs)),
+                               w.image_bytes)
+    bd = torch.zeros(m.n_blocks, dtype=torch.int64, device="cuda")
+    td = torch.zeros(m.n_tensors, dtype=torch.int64, device="cuda")
+    rec = oracle_record(oracle, w)
+    rc, obd, otd = oracle.restore(rec, image_h, np.zeros(w.slab_bytes, np.uint8))
+    assert rc == 0
+
+    def digests_match(want_bd, want_td):
+        torch.cuda.synchronize()
+        assert gms.gms_last_device_status(m) == 0
+        return np.array_equal(bd.cpu().numpy().view(np.uint64), want_bd) and np.array_equal(td.cpu().numpy().view(np.uint64), want_td)
+
+    gms.gms_restore(m, image, gms.SRC_DEVICE, bd, td)
+    assert digests_match(obd, otd)
+    gms.gms_service_commit(svc)
+
+    # detach: the ranges are unmapped (never touched here), the physical memory stays with the service
+    gms.gms_service_detach(svc)
+    assert gms.gms_service_info(svc)["attached"] == 0
+    scratch = torch.empty(64 * MiB, dtype=torch.uint8, device="cuda")  # other allocations come and go meanwhile
+    scratch.fill_(0xAB)
+    del scratch
+    gms.gms_service_reattach(svc)
+    assert not any(gms.gms_service_access(svc, p) for p in ptrs)  # read-only again, same addresses
+    bd.zero_()
+    td.zero_()
+    gms.gms_digest(m, bd, td)
+    assert digests_match(obd, otd)  # contents survived
+
+    # the memory is lost and rebuilt: fresh pages behind the same addresses, refilled from another image
+    gms.gms_service_acquire_rw(svc)
+    gms.gms_service_release_pages(svc)
+    assert gms.gms_service_info(svc)["backed"] == 0
+    gms.gms_service_back_pages(svc)
+    assert all(gms.gms_service_access(svc, p) for p in ptrs)
+    image2_h = W.random_bytes_host(w.image_bytes, seed=213)
+    rc, obd2, otd2 = oracle.restore(rec, image2_h, np.zeros(w.slab_bytes, np.uint8))
+    gms.gms_restore(m, torch.from_numpy(image2_h).cuda(), gms.SRC_DEVICE, bd, td)
+    assert digests_match(obd2, otd2)
+    bd.zero_()
+    td.zero_()
+    gms.gms_digest(m, bd, td)
+    assert digests_match(obd2, otd2)
+    gms.gms_service_commit(svc)
+    m.close()
+    svc.close()
