@@ -234,7 +234,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         m->block_base[n] = acc;
 
         // ---- chunk length (needs the number of warps the restore kernel runs; a B200's if no device is asked)
-        uint32_t total_warps = 148 * 8;
+        uint32_t total_warps = 148 * 9;
         if (!m->host_only) {
             gms::Geometry g;
             cudaError_t e = gms::get_geometry(gms::kRestore, &g);
