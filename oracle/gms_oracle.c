@@ -334,3 +334,42 @@ int gmso_kv_digest(const uint8_t *pool_base, uint64_t plane_stride, uint64_t blo
     if (skipped) *skipped = skip;
     return GMSO_OK;
 }
+
+/*
+ * Paged-KV verify: the trust decision for KV state that outlived an engine (Section 6, "Preserving KV state",
+ * read with the intact-state rule of Section 2.2), in terms a block manager can act on.  computed and expected
+ * are digest arrays laid out as gmso_kv_restore / gmso_kv_digest lay them out, slot (j * n_planes + p) * k + c.
+ * The result is the set of (pool block id, plane, 4 KiB sub-block) whose digests differ, in ascending
+ * (list position j, plane p, sub-block c) order; an id outside [0, n_blocks) was never copied or digested and is
+ * never reported, whatever its slots hold.  Returns the size of the whole set; only the first `cap` members are
+ * written.
+ */
+typedef struct {
+    uint32_t block_id;  /* ids[j]                                   */
+    uint32_t plane;     /* p                                        */
+    uint32_t sub_block; /* c: 4 KiB block inside the KV block       */
+    uint32_t list_pos;  /* j: position of the block in the id list  */
+} gmso_kv_mismatch;
+
+uint64_t gmso_kv_verify(uint32_t n_planes, uint32_t n_blocks, uint32_t block_bytes, const int32_t *ids, uint32_t n_sel,
+                        const uint64_t *computed, const uint64_t *expected, gmso_kv_mismatch *out, uint64_t cap)
+{
+    uint64_t k = block_bytes / GMSO_BLOCK, count = 0;
+    for (uint32_t j = 0; j < n_sel; ++j) {
+        if (ids[j] < 0 || (uint32_t)ids[j] >= n_blocks) continue;
+        for (uint32_t p = 0; p < n_planes; ++p)
+            for (uint64_t c = 0; c < k; ++c) {
+                uint64_t slot = ((uint64_t)j * n_planes + p) * k + c;
+                if (computed[slot] != expected[slot]) {
+                    if (count < cap) {
+                        out[count].block_id = (uint32_t)ids[j];
+                        out[count].plane = p;
+                        out[count].sub_block = (uint32_t)c;
+                        out[count].list_pos = j;
+                    }
+                    ++count;
+                }
+            }
+    }
+    return count;
+}

@@ -25,6 +25,7 @@ ENTRY_DTYPE = np.dtype(
     [("tensor_id", "<u8"), ("src_offset", "<u8"), ("dst_offset", "<u8"), ("nbytes", "<u8")], align=False
 )
 MISMATCH_DTYPE = np.dtype([("tensor_id", "<u8"), ("block", "<u8")], align=False)
+KV_MISMATCH_DTYPE = np.dtype([("block_id", "<u4"), ("plane", "<u4"), ("sub_block", "<u4"), ("list_pos", "<u4")], align=False)
 
 OK, ERR_NULL, ERR_ALIGN, ERR_RANGE, ERR_OVERLAP, ERR_DUP_ID = 0, -1, -2, -3, -4, -5
 BLOCK = 4096
@@ -71,6 +72,8 @@ def lib():
         L.gmso_verify.argtypes = [p, C.c_size_t, p, p, p, u64]
         L.gmso_kv_digest.restype = C.c_int
         L.gmso_kv_digest.argtypes = [p, u64, u64, C.c_uint32, C.c_uint32, C.c_uint32, p, C.c_uint32, p, p, p]
+        L.gmso_kv_verify.restype = u64
+        L.gmso_kv_verify.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32, p, C.c_uint32, p, p, p, u64]
         L.gmso_kv_restore.restype = C.c_int
         L.gmso_kv_restore.argtypes = [p, u64, u64, C.c_uint32, C.c_uint32, C.c_uint32, p, u64, u64, p, C.c_uint32, p, p, p]
         _lib = L
@@ -233,3 +236,19 @@ def kv_digest(pool: np.ndarray, plane_stride: int, block_stride: int, n_planes: 
     rc = lib().gmso_kv_digest(_ptr(pool_b), plane_stride, block_stride, n_planes, n_blocks, block_bytes, _ptr(ids),
                               len(ids), _ptr(bd), _ptr(kd), C.addressof(skipped))
     return int(rc), bd, kd, int(skipped.value)
+
+
+def kv_verify(n_planes: int, n_blocks: int, block_bytes: int, ids: np.ndarray, computed: np.ndarray, expected: np.ndarray,
+              cap: int):
+    """Differing (block_id, plane, sub_block, list_pos) records in (list position, plane, sub-block) order.
+
+    Returns (count, records[:min(count, cap)]).
+    """
+    ids = np.ascontiguousarray(ids, dtype=np.int32)
+    computed = np.ascontiguousarray(computed, dtype=np.uint64)
+    expected = np.ascontiguousarray(expected, dtype=np.uint64)
+    assert computed.size == expected.size == len(ids) * n_planes * (block_bytes // BLOCK)
+    out = np.zeros(max(cap, 1), dtype=KV_MISMATCH_DTYPE)
+    n = int(lib().gmso_kv_verify(n_planes, n_blocks, block_bytes, _ptr(ids), len(ids), _ptr(computed), _ptr(expected),
+                                 _ptr(out), int(cap)))
+    return n, out[: min(n, cap)].copy()

@@ -418,6 +418,57 @@ def test_kv_digest_is_the_tensor_digest_of_the_block_planes_in_place(oracle):
     assert np.nonzero(kd3 != kd)[0].tolist() == [3]
 
 
+def test_kv_verify_agrees_with_byte_comparison_of_pool_blocks_and_image_slots(oracle):
+    """The pin of kv_verify: put an image into a pool, damage pool bytes by hand, and compare what kv_verify names
+    (from the digests of the damaged pool against the digests the restore reported) with a brute-force byte
+    comparison of every pool block against its image slot, 4 KiB at a time, walked in list order."""
+    rng = np.random.default_rng(54)
+    n_planes, n_blocks, bb = 3, 11, 12288
+    k = bb // 4096
+    ids = np.array([7, -3, 2, 10, 11, 0, 5], np.int32)  # -3 and 11 are out of range
+    plane_stride, ips = n_blocks * bb + 256, len(ids) * bb
+    pool = rng.integers(0, 256, n_planes * plane_stride, dtype=np.uint8)
+    image = rng.integers(0, 256, n_planes * ips, dtype=np.uint8)
+    rc, expected, _, skipped = oracle.kv_restore(pool, plane_stride, bb, n_planes, n_blocks, bb, image, ips, bb, ids)
+    assert rc == 0 and skipped == 2
+    rc, computed, _, _ = oracle.kv_digest(pool, plane_stride, bb, n_planes, n_blocks, bb, ids)
+    assert oracle.kv_verify(n_planes, n_blocks, bb, ids, computed, expected, 8)[0] == 0
+    # host-made damage: single bits in chosen (block id, plane, sub-block), plus one in a block that is not in the list
+    damage = [(2, 0, 1), (7, 2, 2), (7, 0, 0), (0, 1, 0), (5, 2, 2), (5, 2, 0)]
+    for blk, p, c in damage:
+        pool[p * plane_stride + blk * bb + c * 4096 + int(rng.integers(0, 4096))] ^= 1 << int(rng.integers(0, 8))
+    pool[1 * plane_stride + 3 * bb + 17] ^= 0xFF  # block 3 is not selected: must not show up
+    rc, computed, _, _ = oracle.kv_digest(pool, plane_stride, bb, n_planes, n_blocks, bb, ids)
+
+    def brute():
+        out = []
+        for j, blk in enumerate(ids):
+            if not 0 <= blk < n_blocks:
+                continue
+            for p in range(n_planes):
+                for c in range(k):
+                    a = pool[p * plane_stride + blk * bb + c * 4096 :][:4096]
+                    b = image[p * ips + j * bb + c * 4096 :][:4096]
+                    if not np.array_equal(a, b):
+                        out.append((int(blk), p, c, j))
+        return out
+
+    want = brute()
+    assert sorted((b, p, c) for b, p, c, _ in want) == sorted(damage)
+    count, recs = oracle.kv_verify(n_planes, n_blocks, bb, ids, computed, expected, 16)
+    assert count == len(want) == 6
+    assert [(int(r["block_id"]), int(r["plane"]), int(r["sub_block"]), int(r["list_pos"])) for r in recs] == want
+    # cap below the count: the total is still reported, the list is cut, its order unchanged
+    count, recs = oracle.kv_verify(n_planes, n_blocks, bb, ids, computed, expected, 4)
+    assert count == 6 and [(int(r["block_id"]), int(r["plane"]), int(r["sub_block"]), int(r["list_pos"])) for r in recs] == want[:4]
+    assert oracle.kv_verify(n_planes, n_blocks, bb, ids, computed, expected, 0)[0] == 6
+    # slots of skipped ids are never reported, whatever they hold
+    noisy = computed.copy()
+    noisy[(1 * n_planes + 0) * k + 0] ^= 1   # list position 1 is id -3
+    noisy[(4 * n_planes + 2) * k + 2] ^= 1   # list position 4 is id 11
+    assert oracle.kv_verify(n_planes, n_blocks, bb, ids, noisy, expected, 16)[0] == 6
+
+
 def test_oracle_has_not_drifted_from_its_stored_outputs(oracle):
     """tests/golden/oracle_regression.txt was written by tests/golden/make_oracle_regression.py, which calls only the
     oracle: a drift alarm (any later change to the oracle's arithmetic must be deliberate), not a correctness pin."""
