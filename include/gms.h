@@ -46,7 +46,10 @@
  *  - Pointers are marked (device), (host) or (device-accessible).  The caller
  *    owns every buffer it passes and keeps it alive until the stream work has
  *    completed.  The library allocates only the manifest's own small tables
- *    (32 bytes per <=128 KiB of payload, plus the recorded digests).
+ *    (by default 32 bytes per 16 KiB of payload -- 31 MB for a 16 GB manifest --
+ *    plus 8 bytes per 4 KiB block once digests have been recorded, and a second
+ *    copy of the 32-byte records, sorted by source offset, once gms_restore_fd
+ *    or gms_restore_staged has been used on the manifest).
  *  - Calls that use the same manifest must not overlap on the GPU (they share
  *    the manifest's work counter and status word); enqueue them on one stream
  *    or order them with events.
@@ -90,12 +93,14 @@ extern "C" {
                                   gms_restore / gms_capture / gms_digest of this manifest the barrier of
                                   the first block of chunk 0 is told to expect 16 bytes that are never
                                   sent, so the warp that claims it gives up after its wait limit (2 s),
-                                  sets GMS_DEV_TIMEOUT, drains its copies and returns; the other warps
-                                  finish their work.  Nothing faults; outputs of that call are
-                                  incomplete by design.                                        */
+                                  sets GMS_DEV_TIMEOUT, waits at most one more limit (2 s in all, not
+                                  per copy) for the copies it still has in flight, and returns: the call
+                                  ends by itself about 4 s after it began; the other warps finish their
+                                  work.  Nothing faults; outputs of that call are incomplete by design. */
 
 /* bits of the device status word */
-#define GMS_DEV_TIMEOUT 1ull   /* a warp gave up waiting for one of its own bulk copies       */
+#define GMS_DEV_TIMEOUT 1ull   /* a warp gave up waiting for one of its own bulk copies (2 s), then
+                                  spent up to 2 s more draining the rest: worst case 4 s per call  */
 
 typedef struct gms_manifest gms_manifest; /* opaque */
 
@@ -117,7 +122,8 @@ typedef struct {
  * commit); Section 3.2 (the allocations it describes).
  * Validates `entries` (host, n of them) against an image of `image_bytes`
  * bytes and builds the work list that gms_restore / gms_digest walk: every
- * tensor is cut into chunks of at most 32 blocks so that thousands of small
+ * tensor is cut into chunks of 4 blocks (16 KiB; fewer for manifests too small
+ * to give every warp two chunks, never more than 32) so that thousands of small
  * and a few huge tensors are served by one persistent launch.
  * Block digests are laid out in entry order: tensor t owns slots
  * [first_block(t), first_block(t) + ceil(nbytes_t/4096)).
@@ -200,6 +206,21 @@ int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_misma
                uint64_t *d_count, void *stream);
 
 /*
+ * gms_digest_verify / gms_restore_verify -- gms_digest (resp. gms_restore) followed by gms_verify, with the
+ * comparison folded into the pass that computes the digests (Section 2.2 and Section 3.2: the intact-state check
+ * sits on the critical path of a reattach, so it should cost no pass of its own).  Outputs are exactly those of
+ * the two separate calls: block and tensor digests, the ordered mismatch list and the total count.  While a
+ * block's digest is still in a register the streaming kernel compares it with the recorded one and counts the
+ * difference against the block's 2048-slot segment; what remains of gms_verify is its ordered emit, one small
+ * kernel.  d_block_digests is required here (the emit pass reads it back for the segments that differ).
+ * Errors: those of gms_digest / gms_restore, and STATE when nothing has been recorded.
+ */
+int gms_digest_verify(const gms_manifest *m, uint64_t *d_block_digests, uint64_t *d_tensor_digests, gms_mismatch *d_out,
+                      uint32_t cap, uint64_t *d_count, void *stream);
+int gms_restore_verify(const gms_manifest *m, const void *image, uint32_t image_kind, uint64_t *d_block_digests,
+                       uint64_t *d_tensor_digests, gms_mismatch *d_out, uint32_t cap, uint64_t *d_count, void *stream);
+
+/*
  * gms_verify_tensors -- the per-tensor summary of the same trust decision (Section 2.2): which
  * tensors may be reused as they are.  d_tensor_counts (device, n u32, entry order) receives for
  * every entry the number of its blocks whose digest differs from the recorded one (0 = intact).
@@ -217,8 +238,8 @@ int gms_verify_tensors(const gms_manifest *m, const uint64_t *d_block_digests, u
  * or disturb, the engine that is serving on the same device.  gms_verify needs a manifest, and
  * building one allocates.  This entry point compares two digest arrays the caller already holds
  * and allocates nothing: no cudaMalloc, no cudaFree, no allocating library call.  Its working
- * tables (per-segment counts and offsets of the ordered compaction) live in a fixed array of about
- * 24 KiB inside the library image, present on every GPU that loads the library until the process
+ * table (the per-segment counts of the ordered compaction) lives in a fixed array of about
+ * 8 KiB inside the library image, present on every GPU that loads the library until the process
  * exits.
  *
  * What it computes.  Exactly what gms_verify reports for a manifest with the single entry
@@ -230,6 +251,11 @@ int gms_verify_tensors(const gms_manifest *m, const uint64_t *d_block_digests, u
  *                           with GMS_ERR_TOO_LARGE before anything is enqueued
  * Rules.  The first call on a device looks up the device address of the fixed array (a one-time
  * set-up with that device current); make that first call before starting any stream capture.
+ * That first call is also when the CUDA runtime loads this library's code and the array onto the
+ * device, which itself takes device memory: a caller that expects the GPU to fill up should make
+ * one warm-up call with n_blocks <= 16384 and one with n_blocks > 16384 (the two sizes run
+ * different kernels) while memory is still available; only calls after that are allocation-free.
+ * The cached address does not survive a cudaDeviceReset of that device.
  * All calls on a device share the one array, which keeps the previous call's contents (each call
  * rewrites what it uses before use): two calls that overlap on the GPU race, so keep them on one
  * stream or order them with events.  Errors: NULL, TOO_LARGE, ARG, CUDA.
@@ -318,6 +344,9 @@ int gms_host_image_free(void *host_ptr);
  * `n_buffers` pinned, device-mapped buffers of `buffer_bytes` each (>= 1 MiB, multiple of 4096) is
  * filled by `n_readers` threads with pread(), and each filled buffer is consumed by the restore
  * kernel (which reads it across the host link, scatters and digests) while the next one is read.
+ * The first gms_restore_fd (or gms_restore_staged) on a manifest builds and uploads a copy of its work list
+ * sorted by source offset: that call allocates device memory and synchronises, so it must not be made
+ * while a stream capture is in progress.
  * gms_restore_fd is synchronous: on return the stream has been synchronised and the outputs hold
  * exactly what gms_restore would have produced from the same bytes (image byte k = file byte
  * file_offset + k).  One restore at a time per pipe.  Errors: NULL, ARG (bad sizes; a chunk larger
@@ -344,7 +373,8 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
  * cudaMemcpyAsync on an internal stream into a ring of `n_buffers` device buffers of `buffer_bytes`
  * each (>= 1 MiB, multiple of 4096), and every landed window is scattered and digested by the
  * restore kernel on the caller's stream while the next one is in flight; all ordering is done with
- * stream events, no kernel waits for a flag.  Asynchronous like gms_restore: outputs are valid once
+ * stream events, no kernel waits for a flag.  Asynchronous like gms_restore (after the first call on a
+ * manifest, which uploads the sorted work list as described above): outputs are valid once
  * `stream` has been synchronised; the host image must stay untouched until then.  Results are
  * exactly those of gms_restore from the same bytes.  `host_image` (host) must be pinned memory.
  * Errors: NULL, ARG, KIND (not pinned host memory), NOMEM, STATE, CUDA.

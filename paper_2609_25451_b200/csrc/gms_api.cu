@@ -29,7 +29,7 @@ struct gms_manifest {
     // device tables (one allocation) and the recorded digests (allocated on first use)
     uint8_t *d_tables = nullptr;
     Chunk *d_chunks = nullptr;
-    uint64_t *d_block_base = nullptr, *d_tensor_ids = nullptr, *d_seg_offset = nullptr;
+    uint64_t *d_block_base = nullptr, *d_tensor_ids = nullptr;
     uint32_t *d_seg_count = nullptr;
     unsigned int *d_counter = nullptr;
     unsigned long long *d_status = nullptr;
@@ -166,6 +166,9 @@ int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void
     a.capture = 0;
     a.keep_accum = first ? 0u : 1u;
     a.stall_chunk = 0xffffffffu;
+    a.expected = nullptr;
+    a.seg_count = nullptr;
+    a.n_segments = 0;
     cudaError_t e = launch_restore(a, s);
     return e == cudaSuccess ? GMS_OK : cuda_fail(e);
 }
@@ -261,8 +264,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             const size_t o_chunks = 0;
             const size_t o_base = align_up(o_chunks + m->chunks.size() * sizeof(Chunk), 256);
             const size_t o_ids = align_up(o_base + (n + 1) * sizeof(uint64_t), 256);
-            const size_t o_segoff = align_up(o_ids + n * sizeof(uint64_t), 256);
-            const size_t o_segcnt = align_up(o_segoff + (size_t)m->n_segments * sizeof(uint64_t), 256);
+            const size_t o_segcnt = align_up(o_ids + n * sizeof(uint64_t), 256);
             const size_t o_ctr = align_up(o_segcnt + (size_t)m->n_segments * sizeof(uint32_t), 256);
             const size_t o_status = o_ctr + (size_t)gms::kMaxCounters * gms::kCounterStride * sizeof(unsigned int);
             const size_t total = o_status + 128;
@@ -285,7 +287,6 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             m->d_chunks = reinterpret_cast<Chunk *>(m->d_tables + o_chunks);
             m->d_block_base = reinterpret_cast<uint64_t *>(m->d_tables + o_base);
             m->d_tensor_ids = reinterpret_cast<uint64_t *>(m->d_tables + o_ids);
-            m->d_seg_offset = reinterpret_cast<uint64_t *>(m->d_tables + o_segoff);
             m->d_seg_count = reinterpret_cast<uint32_t *>(m->d_tables + o_segcnt);
             m->d_counter = reinterpret_cast<unsigned int *>(m->d_tables + o_ctr);
             m->d_status = reinterpret_cast<unsigned long long *>(m->d_tables + o_status);
@@ -364,7 +365,7 @@ int gms_manifest_set_expected(gms_manifest *m, const uint64_t *d_block_digests, 
 }
 
 static int stream_call(const gms_manifest *m, const void *image, bool store, uint64_t *d_block_digests,
-                       uint64_t *d_tensor_digests, void *stream, bool capture = false)
+                       uint64_t *d_tensor_digests, void *stream, bool capture = false, bool compare = false)
 {
     gms::StreamArgs a;
     a.chunks = m->d_chunks;
@@ -381,6 +382,9 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
     a.capture = capture ? 1u : 0u;
     a.keep_accum = 0;
     a.stall_chunk = m->selftest_stall ? 0u : 0xffffffffu;
+    a.expected = compare ? m->d_expected : nullptr;
+    a.seg_count = compare ? m->d_seg_count : nullptr;
+    a.n_segments = compare ? m->n_segments : 0;
     GMS_CUDA(store ? gms::launch_restore(a, static_cast<cudaStream_t>(stream))
                    : gms::launch_digest(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
@@ -435,13 +439,56 @@ int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_misma
     a.tensor_ids = m->d_tensor_ids;
     a.n_tensors = (uint32_t)m->entries.size();
     a.seg_count = m->d_seg_count;
-    a.seg_offset = m->d_seg_offset;
     a.n_segments = m->n_segments;
     a.out = d_out;
     a.cap = cap;
     a.count = d_count;
     GMS_CUDA(gms::launch_verify(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
+}
+
+// The streaming kernel has counted the differing slots of every segment; only the ordered emit is left.
+static int verify_counted(const gms_manifest *m, const uint64_t *d_block_digests, gms_mismatch *d_out, uint32_t cap,
+                          uint64_t *d_count, void *stream)
+{
+    gms::VerifyArgs a;
+    a.computed = d_block_digests;
+    a.expected = m->d_expected;
+    a.n_blocks = m->n_blocks;
+    a.block_base = m->d_block_base;
+    a.tensor_ids = m->d_tensor_ids;
+    a.n_tensors = (uint32_t)m->entries.size();
+    a.seg_count = m->d_seg_count;
+    a.n_segments = m->n_segments;
+    a.out = d_out;
+    a.cap = cap;
+    a.count = d_count;
+    GMS_CUDA(gms::launch_verify_counted(a, static_cast<cudaStream_t>(stream)));
+    return GMS_OK;
+}
+
+int gms_digest_verify(const gms_manifest *m, uint64_t *d_block_digests, uint64_t *d_tensor_digests, gms_mismatch *d_out,
+                      uint32_t cap, uint64_t *d_count, void *stream)
+{
+    if (!m || !d_count || (cap && !d_out) || (m->n_blocks && !d_block_digests)) return GMS_ERR_NULL;
+    if (m->host_only || !m->has_expected) return GMS_ERR_STATE;
+    const int rc = stream_call(m, nullptr, false, d_block_digests, d_tensor_digests, stream, false, true);
+    return rc ? rc : verify_counted(m, d_block_digests, d_out, cap, d_count, stream);
+}
+
+int gms_restore_verify(const gms_manifest *m, const void *image, uint32_t image_kind, uint64_t *d_block_digests,
+                       uint64_t *d_tensor_digests, gms_mismatch *d_out, uint32_t cap, uint64_t *d_count, void *stream)
+{
+    if (!m || (!image && m->payload) || !d_count || (cap && !d_out) || (m->n_blocks && !d_block_digests)) return GMS_ERR_NULL;
+    if (image_kind != GMS_SRC_DEVICE && image_kind != GMS_SRC_HOST_MAPPED) return GMS_ERR_KIND;
+    if (reinterpret_cast<uint64_t>(image) & 15u) return GMS_ERR_ALIGN;
+    if (m->host_only || !m->has_expected) return GMS_ERR_STATE;
+    if (image) {
+        const int rc = check_kind(image, image_kind);
+        if (rc) return rc;
+    }
+    const int rc = stream_call(m, image, true, d_block_digests, d_tensor_digests, stream, false, true);
+    return rc ? rc : verify_counted(m, d_block_digests, d_out, cap, d_count, stream);
 }
 
 int gms_verify_tensors(const gms_manifest *m, const uint64_t *d_block_digests, uint32_t *d_tensor_counts, void *stream)

@@ -57,6 +57,9 @@ struct StreamArgs {
     uint32_t capture;              // 1: gather allocations into the image (restore kernel with roles swapped)
     uint32_t keep_accum;           // 1: a later window of a windowed restore (accumulators and status are kept)
     uint32_t stall_chunk;          // self-test (GMS_BUILD_SELFTEST_STALL): chunk whose first wait runs out; else 0xffffffff
+    const uint64_t *expected;      // fused compare: the recorded block digests (null: no compare)
+    uint32_t *seg_count;           // fused compare: per-segment mismatch counters, cleared by the prologue
+    uint32_t n_segments;
 };
 
 struct KvArgs {
@@ -86,15 +89,17 @@ struct VerifyArgs {
     const uint64_t *block_base;    // n_tensors + 1 prefix sums (device)
     const uint64_t *tensor_ids;    // n_tensors (device)
     uint32_t n_tensors;
-    uint32_t *seg_count;           // n_segments scratch (device)
-    uint64_t *seg_offset;          // n_segments scratch (device)
+    uint32_t *seg_count;           // n_segments scratch (device): differing slots per segment
     uint32_t n_segments;
     void *out;                     // gms_mismatch[cap]
     uint32_t cap;
     uint64_t *count;
 };
-constexpr uint32_t kVerifySegBlocks = 2048;  // digest slots compared by one CTA
+constexpr uint32_t kVerifySegShift = 11;
+constexpr uint32_t kVerifySegBlocks = 1u << kVerifySegShift;  // digest slots compared by one CTA (one counter each)
 cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s);
+// scan + emit only: the per-segment counts have been produced by a streaming kernel's fused compare
+cudaError_t launch_verify_counted(const VerifyArgs &a, cudaStream_t s);
 cudaError_t launch_verify_tensor_counts(const VerifyArgs &a, uint32_t *counts, cudaStream_t s);
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s);
 

@@ -25,11 +25,10 @@ static_assert(kMaxBlocks % gms::kVerifySegBlocks == 0, "capacity must be a whole
 struct Scratch {
     uint64_t block_base[2];             // {0, n_blocks}: the one "tensor" of a flat comparison
     uint64_t tensor_id[2];              // [0] = the id to report; [1] unused
-    uint64_t seg_offset[kMaxSegments];  // exclusive prefix sums of seg_count
     uint32_t seg_count[kMaxSegments];   // differing slots per segment
 };
 
-// ~24 KiB per GPU that loads the library, held until the process exits.
+// ~8 KiB per GPU that loads the library, held until the process exits.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(Scratch)];
 
 // Rewrites the small tables for this call and clears the per-segment words the call will use
@@ -44,10 +43,7 @@ __global__ void gms_noalloc_setup_kernel(uint64_t n_blocks, uint64_t tensor_id, 
         s->tensor_id[0] = tensor_id;
         s->tensor_id[1] = 0;
     }
-    for (uint32_t k = i; k < n_segments; k += gridDim.x * blockDim.x) {
-        s->seg_count[k] = 0;
-        s->seg_offset[k] = 0;
-    }
+    for (uint32_t k = i; k < n_segments; k += gridDim.x * blockDim.x) s->seg_count[k] = 0;
 }
 
 std::mutex g_mu;
@@ -90,7 +86,6 @@ extern "C" int gms_verify_flat_noalloc(const uint64_t *d_computed, const uint64_
     a.tensor_ids = scratch->tensor_id;
     a.n_tensors = 1;
     a.seg_count = scratch->seg_count;
-    a.seg_offset = scratch->seg_offset;
     a.n_segments = n_segments;
     a.out = d_out;
     a.cap = cap;

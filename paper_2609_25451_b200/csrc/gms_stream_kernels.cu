@@ -93,18 +93,22 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Wait for a phase of one of the warp's own barriers; false after kWaitLimitNs.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+// Wait for a phase of one of the warp's own barriers until the global timer passes `deadline`; false if it did.
+__device__ __forceinline__ bool mbar_wait_until(uint32_t bar, uint32_t parity, uint64_t deadline)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
     for (uint32_t outer = 0; outer < (1u << 24); ++outer) {
 #pragma unroll 1
         for (int i = 0; i < 32; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+        if (global_timer_ns() > deadline) return false;
     }
     return false;
+}
+// Wait for a phase of one of the warp's own barriers; false after kWaitLimitNs.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_until(bar, parity, global_timer_ns() + kWaitLimitNs);
 }
 // 1-D bulk copy global -> shared (bytes: multiple of 16, both addresses 16-byte aligned).
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
@@ -136,14 +140,35 @@ __device__ __forceinline__ uint64_t mix_full(uint64_t z)
     z = (z ^ (z >> 27)) * kM2;
     return z ^ (z >> 31);
 }
-// mix(w ^ c) without its last xor-shift; cfold = c ^ (c >> 30).
-__device__ __forceinline__ uint64_t mix_head(uint64_t w, uint64_t cfold)
+// Three-input XOR in one LOP3.
+__device__ __forceinline__ uint32_t xor3(uint32_t a, uint32_t b, uint32_t c)
 {
-    // (two hand-spelled 32-bit versions of this -- products via mul.hi, or via mul.wide with explicit funnel shifts --
-    // executed 2-5 % fewer instructions and ran 4-9 % slower; the compiler's own lowering of the 64-bit form stays)
-    uint64_t z = (w ^ (w >> 30) ^ cfold) * kM1;
-    z = (z ^ (z >> 27)) * kM2;
-    return z;
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// Low 64 bits of (th:tl) * (Mh:Ml): one widening multiply and two multiply-adds.
+__device__ __forceinline__ void mul64_lo(uint32_t tl, uint32_t th, uint32_t Ml, uint32_t Mh, uint32_t &pl, uint32_t &ph)
+{
+    asm("{\n\t.reg .u64 p;\n\tmul.wide.u32 p, %2, %3;\n\tmov.b64 {%0, %1}, p;\n\t}" : "=r"(pl), "=r"(ph) : "r"(tl), "r"(Ml));
+    asm("mad.lo.u32 %0, %1, %2, %0;" : "+r"(ph) : "r"(tl), "r"(Mh));
+    asm("mad.lo.u32 %0, %1, %2, %0;" : "+r"(ph) : "r"(th), "r"(Ml));
+}
+// mix(w ^ c) without its last xor-shift, on 32-bit halves; (cl, ch) = c ^ (c >> 30).
+// Spelled out so that a word costs exactly 2 widening multiplies, 4 multiply-adds, 4 shifts and 4 LOP3 (plus one
+// LOP3 per word for the running XOR): the compiler's lowering of the plain 64-bit form executes 8.5 multiply-pipe
+// and 11.6 ALU instructions per word (register moves, two-input XORs), this one 6.6 and 9.5 -- measured on a
+// block already in shared memory: 11.4 TB/s of payload against 9.8 at 1965 MHz.  Spelling the shifts as
+// multiplies by powers of two (to move them to the multiply pipe) was measured too and is slower (7.0-10.4 TB/s):
+// the widening and high-half multiplies cost the pipe twice what a low-half multiply-add does.
+__device__ __forceinline__ void mix_head32(uint32_t lo, uint32_t hi, uint32_t cl, uint32_t ch, uint32_t &ql, uint32_t &qh)
+{
+    constexpr uint32_t M1l = (uint32_t)kM1, M1h = (uint32_t)(kM1 >> 32), M2l = (uint32_t)kM2, M2h = (uint32_t)(kM2 >> 32);
+    const uint32_t tl = xor3(lo, __funnelshift_r(lo, hi, 30), cl), th = xor3(hi, hi >> 30, ch);
+    uint32_t zl, zh;
+    mul64_lo(tl, th, M1l, M1h, zl, zh);
+    const uint32_t ul = zl ^ __funnelshift_r(zl, zh, 27), uh = zh ^ (zh >> 27);
+    mul64_lo(ul, uh, M2l, M2h, ql, qh);
 }
 __device__ __forceinline__ uint64_t warp_xor64(uint64_t v)
 {
@@ -240,9 +265,9 @@ struct ListProvider {
             draw(lane);
         }
     }
-    __device__ __forceinline__ void init(uint32_t lane, uint32_t gwarp)
+    __device__ __forceinline__ void init(uint32_t lane)
     {
-        home = gwarp % n_counters;
+        home = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) % n_counters;
         exhausted = 0;
         raw_next = 0;
         grp_left = 0;
@@ -330,9 +355,14 @@ struct KvProvider {
 };
 
 // ---------------------------------------------------------------- the per-warp pipeline
+// `expected` / `seg_count` (both null, or both set): the fused compare.  At the end of a chunk every lane that holds
+// a block digest checks it against the recorded one and, if they differ, bumps the counter of the 2048-slot
+// segment the block lies in -- the first pass of the ordered compaction in gms_verify_kernels.cu, done here
+// while the digest is still in a register, so that gms_digest_verify / gms_restore_verify only run scan + emit.
 template <int S, bool kStore, class Provider>
 __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint4 *fifo, uint64_t *bars, uint64_t *block_digests,
-                                             uint64_t *accum, unsigned long long *status, uint32_t hints)
+                                             uint64_t *accum, unsigned long long *status, uint32_t hints,
+                                             const uint64_t *expected, uint32_t *seg_count)
 {
     static_assert(S <= (int)kFifo, "the chunk fifo must cover the ring");
     constexpr uint32_t LOOK = S - 1;  // blocks in flight ahead of the one being digested
@@ -340,13 +370,14 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
 
     // folded position constants of the 16 words this lane sees in every block:
     // 16-byte load j (0..7) of lane l covers words 64 j + 2 l and 64 j + 2 l + 1.
-    uint64_t cfold[16];
+    uint32_t cl[16], ch[16];
 #pragma unroll
     for (int j = 0; j < 8; ++j)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-            const uint64_t c = (uint64_t)(64 * j + 2 * lane + e) * kG;
-            cfold[2 * j + e] = c ^ (c >> 30);
+            const uint64_t c = (uint64_t)(64 * j + 2 * lane + e) * kG, f = c ^ (c >> 30);
+            cl[2 * j + e] = (uint32_t)f;
+            ch[2 * j + e] = (uint32_t)(f >> 32);
         }
 
     const uint32_t ring_s = smem_u32(ring), bars_s = smem_u32(bars);
@@ -358,6 +389,11 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
         fence_mbar_init();
     }
     __syncwarp();
+    // Everything above touched registers and this warp's own shared memory only, so it ran while the grid before
+    // this one (the prologue that clears counters and accumulators, or whatever the caller enqueued) was still
+    // running.  From here on global memory is read and written: wait for that grid's writes.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    prov.init(lane);
 
     // issue-side cursor (the chunk being fetched) and digest-side cursor (the chunk being consumed);
     // chunk records travel from one to the other through a small per-warp fifo in shared memory
@@ -457,19 +493,24 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
             }
             bulk_commit();
         }
-        uint64_t acc = 0;
+        uint32_t al = 0, ah = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint4 v = *reinterpret_cast<const uint4 *>(stage + 512 * j + 16 * lane);
-            acc ^= mix_head(((uint64_t)v.y << 32) | v.x, cfold[2 * j]) ^ mix_head(((uint64_t)v.w << 32) | v.z, cfold[2 * j + 1]);
+            uint32_t pl, ph, ql, qh;
+            mix_head32(v.x, v.y, cl[2 * j], ch[2 * j], pl, ph);
+            mix_head32(v.z, v.w, cl[2 * j + 1], ch[2 * j + 1], ql, qh);
+            al = xor3(al, pl, ql);
+            ah = xor3(ah, ph, qh);
         }
-        acc = warp_xor64(acc);
+        const uint64_t acc = ((uint64_t)__reduce_xor_sync(kFull, ah) << 32) | __reduce_xor_sync(kFull, al);
         if (lane == c_next) myD = acc ^ (acc >> 31);
         ++c_next;
         if (c_next == c_blocks) {  // chunk complete: block digests leave coalesced, one atomic for the tensor digest
             uint64_t t = 0;
             if (lane < c_blocks) {
                 if (block_digests) block_digests[(uint64_t)c_gblock0 + lane] = myD;
+                if (expected && __ldg(expected + c_gblock0 + lane) != myD) atomicAdd(seg_count + ((c_gblock0 + lane) >> kVerifySegShift), 1u);
                 t = mix_full(myD ^ ((uint64_t)(c_tblock0 + lane) * kG));
             }
             t = warp_xor64(t);
@@ -489,8 +530,9 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
         atomicXor(reinterpret_cast<unsigned long long *>(accum + run_tensor), (unsigned long long)run_val);
     if (failed) {
         if (lane == 0) atomicOr(status, kDevTimeout);
-        // bounded drain of what is still in flight into this warp's ring
-        for (uint32_t b = consumed; b != issued; ++b) (void)mbar_wait_bounded(bars_s + 8u * (b % S), (b / S) & 1u);
+        // drain what is still in flight into this warp's ring, all of it against one more wait limit
+        const uint64_t deadline = global_timer_ns() + kWaitLimitNs;
+        for (uint32_t b = consumed; b != issued; ++b) (void)mbar_wait_until(bars_s + 8u * (b % S), (b / S) & 1u, deadline);
     }
     if (kStore && lane == 0) bulk_wait_all();
 }
@@ -513,8 +555,14 @@ __device__ __forceinline__ SmemLayout carve(uint8_t *smem)
     return l;
 }
 
+// The digest-only shape may run up to 18 warps (its slots are small and it holds no store state).
+#ifdef GMS_EXP_MAXNREG
+#define GMS_STREAM_BOUNDS __maxnreg__(112)
+#else
+#define GMS_STREAM_BOUNDS __launch_bounds__(kStore ? 512 : 576, 1)
+#endif
 template <int S, bool kStore>
-__global__ void __launch_bounds__(512, 1) gms_stream_kernel(StreamArgs a)
+__global__ void GMS_STREAM_BOUNDS gms_stream_kernel(StreamArgs a)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const SmemLayout l = carve<S>(smem);
@@ -527,13 +575,15 @@ __global__ void __launch_bounds__(512, 1) gms_stream_kernel(StreamArgs a)
     prov.image = kStore ? a.image : nullptr;
     prov.capture = kStore && a.capture;
     prov.stall_chunk = a.stall_chunk;
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // the prologue's zeroed counters and accumulators are visible from here
-    prov.init(threadIdx.x & 31u, blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5));
-    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.hints);
+    // whatever follows on the stream may be scheduled now; every kernel of this library waits (griddepcontrol.wait)
+    // for the grid before it to finish before it touches global memory
+    asm volatile("griddepcontrol.launch_dependents;");
+    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.hints, a.expected,
+                            a.seg_count);
 }
 
 template <int S, bool kStore>
-__global__ void __launch_bounds__(512, 1) gms_kv_stream_kernel(KvArgs a)
+__global__ void GMS_STREAM_BOUNDS gms_kv_stream_kernel(KvArgs a)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const SmemLayout l = carve<S>(smem);
@@ -541,21 +591,26 @@ __global__ void __launch_bounds__(512, 1) gms_kv_stream_kernel(KvArgs a)
     prov.a = a;
     prov.counter = reinterpret_cast<unsigned int *>(a.status + 2);
     prov.total = a.n_sel * a.n_planes;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    prov.init(threadIdx.x & 31u);
-    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, a.hints);
+    asm volatile("griddepcontrol.launch_dependents;");
+    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, a.hints, nullptr, nullptr);
 }
 
-// Clears the accumulators the streaming kernels XOR / add into.
+// Clears the accumulators the streaming kernels XOR / add into (and, for the fused compare, the per-segment
+// mismatch counters).
 __global__ void gms_prologue_kernel(uint64_t *accum, uint64_t n_accum, unsigned int *counters, uint32_t n_counters,
-                                    unsigned long long *status, uint32_t n_status)
+                                    unsigned long long *status, uint32_t n_status, uint32_t *seg_count, uint32_t n_segments)
 {
     // let the streaming kernel that follows be scheduled now: it sets itself up (constants, barriers) while this
     // grid runs, and waits (griddepcontrol.wait) for this grid's writes before it touches a counter
     asm volatile("griddepcontrol.launch_dependents;");
+    // this grid may itself have been scheduled early, behind a kernel of this library that is still using the
+    // counters: wait for it before clearing anything
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint64_t i0 = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x, step = (uint64_t)gridDim.x * blockDim.x;
     if (accum)
         for (uint64_t i = i0; i < n_accum; i += step) accum[i] = 0;
+    if (seg_count)
+        for (uint64_t i = i0; i < n_segments; i += step) seg_count[i] = 0;
     if (i0 < n_counters) counters[i0 * kCounterStride] = 0;
     if (i0 < n_status) status[i0] = 0;
 }
@@ -565,7 +620,7 @@ void env_geom(const char *name, uint32_t &w, uint32_t &s, uint32_t &c)
 {
     const char *v = getenv(name);
     unsigned a = 0, b = 0, d = 0;
-    if (v && sscanf(v, "%u,%u,%u", &a, &b, &d) == 3 && a >= 1 && a <= 16 && (b == 3 || b == 4 || b == 6 || b == 8) && d >= 1 && d <= 4) {
+    if (v && sscanf(v, "%u,%u,%u", &a, &b, &d) == 3 && a >= 1 && a <= 18 && (b == 3 || b == 4 || b == 6 || b == 8) && d >= 1 && d <= 4) {
         w = a;
         s = b;
         c = d;
@@ -586,16 +641,33 @@ constexpr int kMaxDevices = 64;
 Geometry g_geom[kMaxDevices][kKinds];
 bool g_geom_ok[kMaxDevices][kKinds];
 
+// Launch attribute shared by every kernel of the library: the grid may be scheduled while its predecessor on the
+// stream still runs (programmatic dependent launch); each kernel waits for the predecessor itself.
+cudaLaunchConfig_t pdl_config(dim3 grid, dim3 block, size_t smem, cudaStream_t s, cudaLaunchAttribute *attr)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cfg;
+}
+
 cudaError_t prologue(uint64_t *accum, uint64_t n_accum, unsigned int *counters, uint32_t n_counters, unsigned long long *status,
-                     uint32_t n_status, cudaStream_t s)
+                     uint32_t n_status, uint32_t *seg_count, uint32_t n_segments, cudaStream_t s)
 {
     const uint32_t threads = 256;
-    uint64_t blocks = accum ? (n_accum + threads - 1) / threads : 1;
+    uint64_t blocks = std::max<uint64_t>(accum ? (n_accum + threads - 1) / threads : 1, seg_count ? (n_segments + threads - 1) / threads : 1);
     if (blocks < 1) blocks = 1;
     if (blocks > 1184) blocks = 1184;
-    gms_prologue_kernel<<<(uint32_t)blocks, threads, 0, s>>>(accum, n_accum, counters, n_counters, status, n_status);
+    cudaLaunchAttribute attr[1];
+    cudaLaunchConfig_t cfg = pdl_config(dim3((uint32_t)blocks), dim3(threads), 0, s, attr);
     count_launches(1);
-    return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, gms_prologue_kernel, accum, n_accum, counters, n_counters, status, n_status, seg_count, n_segments);
 }
 
 // A streaming kernel is always enqueued right behind its prologue.  Programmatic dependent launch lets the
@@ -604,16 +676,8 @@ cudaError_t prologue(uint64_t *accum, uint64_t n_accum, unsigned int *counters, 
 template <class Args>
 cudaError_t launch_after_prologue(void (*kernel)(Args), const Geometry &g, cudaStream_t s, const Args &args)
 {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(g.grid);
-    cfg.blockDim = dim3(g.warps * 32);
-    cfg.dynamicSmemBytes = g.smem;
-    cfg.stream = s;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cudaLaunchConfig_t cfg = pdl_config(dim3(g.grid), dim3(g.warps * 32), g.smem, s, attr);
     return cudaLaunchKernelEx(&cfg, kernel, args);
 }
 
@@ -625,7 +689,7 @@ cudaError_t launch_stream(const StreamArgs &a, cudaStream_t s)
     if (e) return e;
     // a windowed restore keeps the tensor-digest accumulators and the status word of its earlier windows
     if ((e = prologue(a.keep_accum ? nullptr : a.tensor_digests, a.n_tensors, a.work_counters, g.counters, a.status,
-                      a.keep_accum ? 0 : 1, s)))
+                      a.keep_accum ? 0 : 1, a.keep_accum ? nullptr : a.seg_count, a.n_segments, s)))
         return e;
     if (a.n_chunks == 0) return cudaSuccess;
     StreamArgs b = a;
@@ -710,7 +774,7 @@ cudaError_t launch_kv_restore(const KvArgs &a, cudaStream_t s)
     Geometry g;
     cudaError_t e = get_geometry(a.digest_only ? kKvDigest : kKv, &g);
     if (e) return e;
-    if ((e = prologue(a.kv_digests, a.n_sel, nullptr, 0, a.status, 4, s))) return e;
+    if ((e = prologue(a.kv_digests, a.n_sel, nullptr, 0, a.status, 4, nullptr, 0, s))) return e;
     if (a.n_sel == 0 || a.n_planes == 0) return cudaSuccess;
     KvArgs b = a;
     b.hints = g.hints;

@@ -2,11 +2,15 @@
 // the differing (tensor_id, block) pairs in ascending (entry position, block)
 // order.  The order is made deterministic by an ordered compaction instead of
 // an atomic append: (1) every CTA counts the differences in its own contiguous
-// segment of digest slots, (2) one CTA turns the per-segment counts into
-// offsets and the grand total, (3) every CTA whose segment has differences
-// (normally none) ranks them with a block-wide scan and writes them at
-// offset + rank.  Traffic is 16 bytes per 4 KiB of payload -- noise next to the
-// streaming kernels -- and no CTA ever waits for another.
+// segment of 2048 digest slots (or a streaming kernel has already counted them
+// while it held each digest in a register: the fused compare), (2) every CTA
+// whose segment has differences (normally none) adds up the counts of the
+// segments before it -- a few kilobytes out of L2 -- ranks its own differences
+// with a block-wide scan and writes them at offset + rank; the last CTA also
+// writes the grand total.  Traffic is 16 bytes per 4 KiB of payload -- noise
+// next to the streaming kernels -- and no CTA ever waits for another.
+// Every kernel here may be scheduled while its predecessor on the stream still
+// runs (programmatic dependent launch) and waits for it before reading.
 #include "gms_internal.h"
 
 namespace gms {
@@ -33,7 +37,8 @@ __device__ __forceinline__ uint32_t diff_mask(const uint64_t *c, const uint64_t 
 
 __global__ void __launch_bounds__(kThreads) gms_verify_count_kernel(VerifyArgs a)
 {
-    asm volatile("griddepcontrol.launch_dependents;");  // the scan kernel may be scheduled; it waits for our counts
+    asm volatile("griddepcontrol.launch_dependents;");  // the emit kernel may be scheduled; it waits for our counts
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the digests being compared are complete and visible
     __shared__ uint32_t warp_sum[kThreads / 32];
     // only the segment's total matters here, so the slots are read coalesced (16-byte pairs, neighbouring lanes
     // neighbouring pairs); the emit pass, which needs ranks, uses the thread-contiguous layout
@@ -62,45 +67,36 @@ __global__ void __launch_bounds__(kThreads) gms_verify_count_kernel(VerifyArgs a
     }
 }
 
-// One CTA: exclusive prefix sum of the segment counts, and the total.
-__global__ void __launch_bounds__(1024) gms_verify_scan_kernel(VerifyArgs a)
-{
-    __shared__ uint64_t warp_tot[32];
-    __shared__ uint64_t carry;
-    asm volatile("griddepcontrol.launch_dependents;");
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // the per-segment counts are complete and visible
-    if (threadIdx.x == 0) carry = 0;
-    __syncthreads();
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (uint32_t base = 0; base < a.n_segments; base += blockDim.x) {
-        const uint32_t i = base + threadIdx.x;
-        const uint64_t v = i < a.n_segments ? a.seg_count[i] : 0;
-        uint64_t incl = v;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint64_t o = __shfl_up_sync(0xffffffffu, incl, d);
-            if ((int)lane >= d) incl += o;
-        }
-        if (lane == 31) warp_tot[warp] = incl;
-        __syncthreads();
-        uint64_t before = carry;
-        for (uint32_t w = 0; w < warp; ++w) before += warp_tot[w];
-        if (i < a.n_segments) a.seg_offset[i] = before + incl - v;
-        __syncthreads();
-        if (threadIdx.x == blockDim.x - 1) carry = before + incl;
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) *a.count = carry;
-}
-
+// Ordered emit.  CTA k owns segment k.  Its offset in the output is the sum of the counts of segments 0..k-1,
+// which it adds up itself (at most a few thousand 32-bit words, read by 256 threads); segments without
+// differences return at once, except the last one, which also publishes the total.
 __global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
 {
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // counts (first pass) and offsets (scan) are complete
-    if (a.seg_count[blockIdx.x] == 0) return;  // the common case: nothing differs here
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the per-segment counts are complete and visible
+    __shared__ uint64_t warp_tot[kThreads / 32];
     __shared__ uint32_t warp_sum[kThreads / 32];
+    if (a.n_segments == 0) {  // no digest slots at all
+        if (threadIdx.x == 0) *a.count = 0;
+        return;
+    }
+    const bool last = blockIdx.x + 1 == a.n_segments;
+    const uint32_t own = a.seg_count[blockIdx.x];
+    if (own == 0 && !last) return;  // the common case: nothing differs here
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint64_t before = 0;
+    for (uint32_t i = threadIdx.x; i < blockIdx.x; i += kThreads) before += a.seg_count[i];
+#pragma unroll
+    for (int d = 16; d; d >>= 1) before += __shfl_xor_sync(0xffffffffu, before, d);
+    if (lane == 0) warp_tot[warp] = before;
+    __syncthreads();
+    before = 0;
+    for (uint32_t w = 0; w < kThreads / 32; ++w) before += warp_tot[w];
+    if (last && threadIdx.x == 0) *a.count = before + own;
+    if (own == 0) return;
     const uint64_t first = (uint64_t)blockIdx.x * kVerifySegBlocks + (uint64_t)threadIdx.x * kPerThread;
     const uint32_t mask = diff_mask(a.computed, a.expected, first, a.n_blocks);
-    const uint32_t mine = __popc(mask), lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t mine = __popc(mask);
     uint32_t incl = mine;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -109,7 +105,7 @@ __global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
     }
     if (lane == 31) warp_sum[warp] = incl;
     __syncthreads();
-    uint64_t rank = a.seg_offset[blockIdx.x] + incl - mine;
+    uint64_t rank = before + incl - mine;
     for (uint32_t w = 0; w < warp; ++w) rank += warp_sum[w];
     if (!mask) return;
     Mismatch *out = static_cast<Mismatch *>(a.out);
@@ -136,6 +132,8 @@ constexpr uint64_t kSmallBlocks = 16384;
 __global__ void __launch_bounds__(kSmallThreads) gms_verify_small_kernel(VerifyArgs a)
 {
     __shared__ uint32_t warp_sum[kSmallThreads / 32];
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint64_t per = (a.n_blocks + kSmallThreads - 1) / kSmallThreads;  // consecutive slots per thread
     const uint64_t lo = (uint64_t)threadIdx.x * per, hi = lo + per < a.n_blocks ? lo + per : a.n_blocks;
     uint32_t mine = 0;
@@ -174,45 +172,48 @@ __global__ void __launch_bounds__(kSmallThreads) gms_verify_small_kernel(VerifyA
 
 __global__ void gms_copy_u64_kernel(uint64_t *dst, const uint64_t *src, uint64_t n)
 {
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint64_t step = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += step) dst[i] = src[i];
 }
 
 }  // namespace
 
-cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
+namespace {
+template <class... P, class... A>
+cudaError_t launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, cudaStream_t s, A... args)
 {
-    if (a.n_segments == 0) {  // no digest slots at all: count = 0
-        VerifyArgs z = a;
-        gms_verify_scan_kernel<<<1, 32, 0, s>>>(z);
-        count_launches(1);
-        return cudaGetLastError();
-    }
-    if (a.n_blocks <= kSmallBlocks) {
-        gms_verify_small_kernel<<<1, kSmallThreads, 0, s>>>(a);
-        count_launches(1);
-        return cudaGetLastError();
-    }
-    gms_verify_count_kernel<<<a.n_segments, kThreads, 0, s>>>(a);
-    cudaError_t e = cudaGetLastError();
-    if (e) return e;
-    // scan and emit are scheduled while their predecessor still runs (programmatic dependent launch); each
-    // waits for the predecessor's results before reading them
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cfg.gridDim = dim3(1);
-    cfg.blockDim = dim3(1024);
-    if ((e = cudaLaunchKernelEx(&cfg, gms_verify_scan_kernel, a))) return e;
-    cfg.gridDim = dim3(a.n_segments);
-    cfg.blockDim = dim3(kThreads);
-    e = cudaLaunchKernelEx(&cfg, gms_verify_emit_kernel, a);
-    count_launches(3);
-    return e;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+}  // namespace
+
+cudaError_t launch_verify_counted(const VerifyArgs &a, cudaStream_t s)
+{
+    count_launches(1);
+    return launch_pdl(gms_verify_emit_kernel, dim3(a.n_segments ? a.n_segments : 1), dim3(kThreads), s, a);
+}
+
+cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
+{
+    if (a.n_segments == 0) return launch_verify_counted(a, s);  // no digest slots at all: count = 0
+    if (a.n_blocks <= kSmallBlocks) {
+        count_launches(1);
+        return launch_pdl(gms_verify_small_kernel, dim3(1), dim3(kSmallThreads), s, a);
+    }
+    count_launches(1);
+    cudaError_t e = launch_pdl(gms_verify_count_kernel, dim3(a.n_segments), dim3(kThreads), s, a);
+    if (e) return e;
+    return launch_verify_counted(a, s);
 }
 
 namespace {
@@ -222,6 +223,8 @@ namespace {
 // differing slot looks its tensor up and bumps that counter.
 __global__ void gms_verify_tensor_counts_kernel(VerifyArgs a, uint32_t *counts)
 {
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the zeroed counters and the digests are visible
     const uint64_t step = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t g = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; g < a.n_blocks; g += step) {
         if (a.computed[g] == a.expected[g]) continue;
@@ -237,6 +240,7 @@ __global__ void gms_verify_tensor_counts_kernel(VerifyArgs a, uint32_t *counts)
 __global__ void gms_zero_u32_kernel(uint32_t *p, uint64_t n)
 {
     asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint64_t step = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += step) p[i] = 0;
 }
@@ -247,16 +251,14 @@ cudaError_t launch_verify_tensor_counts(const VerifyArgs &a, uint32_t *counts, c
 {
     if (a.n_tensors == 0) return cudaSuccess;
     uint32_t zb = (a.n_tensors + 255) / 256;
-    gms_zero_u32_kernel<<<zb > 592 ? 592 : zb, 256, 0, s>>>(counts, a.n_tensors);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(gms_zero_u32_kernel, dim3(zb > 592 ? 592 : zb), dim3(256), s, counts, (uint64_t)a.n_tensors);
     if (e) return e;
     count_launches(1);
     if (a.n_blocks == 0) return cudaSuccess;
     uint64_t blocks = (a.n_blocks + 1023) / 1024;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    gms_verify_tensor_counts_kernel<<<(uint32_t)blocks, 256, 0, s>>>(a, counts);
     count_launches(1);
-    return cudaGetLastError();
+    return launch_pdl(gms_verify_tensor_counts_kernel, dim3((uint32_t)blocks), dim3(256), s, a, counts);
 }
 
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s)
@@ -264,9 +266,8 @@ cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cuda
     if (n == 0) return cudaSuccess;
     uint64_t blocks = (n + 1023) / 1024;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    gms_copy_u64_kernel<<<(uint32_t)blocks, 256, 0, s>>>(dst, src, n);
     count_launches(1);
-    return cudaGetLastError();
+    return launch_pdl(gms_copy_u64_kernel, dim3((uint32_t)blocks), dim3(256), s, dst, src, n);
 }
 
 }  // namespace gms

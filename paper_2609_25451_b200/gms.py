@@ -33,7 +33,7 @@ MISMATCH_DTYPE = np.dtype([("tensor_id", "<u8"), ("block", "<u8")])
 EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
-    "gms_verify", "gms_verify_tensors", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_kv_digest", "gms_host_image_alloc", "gms_host_image_free",
+    "gms_verify", "gms_digest_verify", "gms_restore_verify", "gms_verify_tensors", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_kv_digest", "gms_host_image_alloc", "gms_host_image_free",
     "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd", "gms_stage_create", "gms_stage_destroy", "gms_restore_staged",
     "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
     "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
@@ -84,6 +84,8 @@ def lib():
             "gms_capture": (i, [p, p, u32, p, p, p]),
             "gms_digest": (i, [p, p, p, p]),
             "gms_verify": (i, [p, p, p, u32, p, p]),
+            "gms_digest_verify": (i, [p, p, p, p, u32, p, p]),
+            "gms_restore_verify": (i, [p, p, u32, p, p, p, u32, p, p]),
             "gms_verify_tensors": (i, [p, p, p, p]),
             "gms_verify_flat_noalloc": (i, [p, p, u64, u64, p, u32, p, p]),
             "gms_last_device_status": (i, [p, p, pu64]),
@@ -221,6 +223,17 @@ def gms_digest(m: Manifest, d_block_digests, d_tensor_digests, stream=None):
 
 def gms_verify(m: Manifest, d_block_digests, d_out, cap: int, d_count, stream=None):
     _check(lib().gms_verify(m.handle, _dev(d_block_digests), _dev(d_out), cap, _dev(d_count), _stream(stream)), "gms_verify")
+
+
+def gms_digest_verify(m: Manifest, d_block_digests, d_tensor_digests, d_out, cap: int, d_count, stream=None):
+    _check(lib().gms_digest_verify(m.handle, _dev(d_block_digests), _dev(d_tensor_digests), _dev(d_out), cap, _dev(d_count),
+                                   _stream(stream)), "gms_digest_verify")
+
+
+def gms_restore_verify(m: Manifest, image, image_kind: int, d_block_digests, d_tensor_digests, d_out, cap: int, d_count,
+                       stream=None):
+    _check(lib().gms_restore_verify(m.handle, _dev(image), image_kind, _dev(d_block_digests), _dev(d_tensor_digests),
+                                    _dev(d_out), cap, _dev(d_count), _stream(stream)), "gms_restore_verify")
 
 
 def gms_verify_tensors(m: Manifest, d_block_digests, d_tensor_counts, stream=None):

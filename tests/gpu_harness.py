@@ -82,6 +82,24 @@ class DeviceWorkload:
         assert (pairs[k:] == CANARY).all(), "verify wrote past min(count, cap)"
         return count, [(int(a), int(b)) for a, b in pairs[:k]]
 
+    def fused(self, cap: int, restore: bool = False):
+        """gms_digest_verify (or gms_restore_verify from the device image): digests, count and mismatch pairs."""
+        self.reset_outputs()
+        out = torch.full((2 * cap + 2 * PAD,), CANARY, dtype=torch.int64, device="cuda")
+        cnt = guarded_u64(1)
+        if restore:
+            gms.gms_restore_verify(self.m, self.image, gms.SRC_DEVICE, self.bd_ptr(), self.td_ptr(), out.data_ptr() + 8 * PAD, cap,
+                                   cnt.data_ptr() + 8 * PAD)
+        else:
+            gms.gms_digest_verify(self.m, self.bd_ptr(), self.td_ptr(), out.data_ptr() + 8 * PAD, cap, cnt.data_ptr() + 8 * PAD)
+        torch.cuda.synchronize()
+        assert gms.gms_last_device_status(self.m) == 0
+        count = int(payload_of(cnt, 1)[0])
+        pairs = payload_of(out, 2 * cap).reshape(cap, 2)
+        k = min(count, cap)
+        assert (pairs[k:] == CANARY).all(), "the fused verify wrote past min(count, cap)"
+        return payload_of(self.bd, self.nb), payload_of(self.td, self.nt), count, [(int(a), int(b)) for a, b in pairs[:k]]
+
     def slab_host(self) -> np.ndarray:
         return self.slab.cpu().numpy()
 

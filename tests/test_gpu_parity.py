@@ -76,6 +76,18 @@ def test_restore_digest_verify_parity(oracle, name):
     assert count == 3 and pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm][:2]
     count, pairs = d.verify(cap=0)
     assert count == 3 and pairs == []
+    # the fused calls: same digests, same list, same count as the oracle's digest + verify
+    want_pairs = [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+    for cap in (8, 2, 0):
+        fbd, ftd, count, pairs = d.fused(cap)
+        assert np.array_equal(fbd, obd3) and np.array_equal(ftd, otd3)
+        assert count == 3 and pairs == want_pairs[:cap]
+    assert np.array_equal(d.slab_host(), want_slab)
+    # restore + verify in one pass: the flips are overwritten, nothing differs any more
+    clean_slab, _, _ = oracle_restore(oracle, w, image)
+    fbd, ftd, count, pairs = d.fused(8, restore=True)
+    assert np.array_equal(fbd, want_bd) and np.array_equal(ftd, want_td) and (count, pairs) == (0, [])
+    assert np.array_equal(d.slab_host(), clean_slab)
     d.close()
 
 
@@ -103,6 +115,7 @@ def test_empty_manifests(oracle):
         assert (td == 0).all()
         gms.gms_manifest_set_expected(d.m, d.bd_ptr())
         assert d.verify(cap=4) == (0, [])
+        assert d.fused(4)[2:] == (0, []) and d.fused(4, restore=True)[2:] == (0, [])
         assert (d.slab_host() == FILL).all()
         d.close()
 
@@ -157,6 +170,17 @@ def test_many_mismatches_exceed_cap_in_order(oracle, scale):
         ocount, omm = oracle.verify(rec, obd, want_bd, cap=cap)
         assert count == ocount and count > 2500
         assert pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+        fbd, _, fcount, fpairs = d.fused(cap)  # the compare folded into the digest pass
+        assert np.array_equal(fbd, obd) and fcount == ocount and fpairs == pairs
+    # restore + verify against digests recorded from the damaged state: every block that was damaged now differs
+    gms.gms_manifest_set_expected(d.m, d.bd_ptr())
+    fbd, _, fcount, fpairs = d.fused(5000, restore=True)
+    ocount2, omm2 = oracle.verify(rec, want_bd, obd, cap=5000)
+    assert np.array_equal(fbd, want_bd) and fcount == ocount2 == ocount
+    assert fpairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm2]
+    d.slab.copy_(torch.from_numpy(want_slab))
+    gms.gms_manifest_set_expected(d.m, torch.from_numpy(want_bd.view(np.int64)).cuda())
+    bd, _ = d.digest()
     # the computed digests may sit at an address that is only 8-byte aligned
     shifted = torch.zeros(d.nb + 1, dtype=torch.int64, device="cuda")
     shifted[1:] = d.bd[PAD:PAD + d.nb]
