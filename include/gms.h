@@ -293,7 +293,11 @@ typedef struct {
  *   d_kv_digests[j] = XOR_q mix(D_q ^ q*G), q = p*k + c  (the tensor digest of
  *                                            the slot's planes concatenated).
  * An id outside [0, n_blocks) is skipped: nothing is written to the pool, its
- * digests are 0, and d_status[0] counts it.  d_status[1] receives the device
+ * digests are 0, and d_status[0] counts it.  With more than one plane,
+ * plane_stride must be at least (n_blocks-1)*block_stride + block_bytes
+ * (planes that share bytes are refused with GMS_ERR_ARG).  That the image
+ * extent covers every slot addressed, and that image and pool do not overlap,
+ * is the caller's duty: the library cannot see the size of either buffer.  d_status[1] receives the device
  * status word; d_status[2..3] are scratch for the kernel's work counter.  Ids
  * must be distinct (the caller's duty; duplicates race).
  *   image        (device-accessible) as for gms_restore; strides multiples of 16
@@ -323,11 +327,39 @@ int gms_kv_capture(const gms_kv_pool *pool, void *image, uint64_t img_plane_stri
  * for every plane p; nothing is written to the pool and there is no image.  Digest layout, skipping
  * of out-of-range ids (digests 0, counted in d_status[0]) and status words are those of
  * gms_kv_restore, so the output compares directly with what gms_kv_restore / gms_kv_capture of the
- * same id list reported (gms_verify_flat_noalloc names the differing 4 KiB blocks).
+ * same id list reported (gms_kv_verify names the differing blocks, planes and 4 KiB sub-blocks).
  * pool->flags is ignored apart from the range check.  Errors: NULL, ALIGN, ARG, RANGE, CUDA.
  */
 int gms_kv_digest(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
                   uint64_t *d_kv_digests, uint64_t *d_status, void *stream);
+
+/*
+ * gms_kv_verify -- the trust decision for preserved KV state (Section 6, "Preserving KV state", read with
+ * Section 2.2: state that outlived an engine is reused only if it is intact), in the terms a block manager acts
+ * on.  d_computed and d_expected (device, n_sel*n_planes*k u64 each, the layout every gms_kv_* call writes:
+ * slot (j*n_planes + p)*k + c) are compared -- typically what gms_kv_digest finds now against what
+ * gms_kv_restore / gms_kv_capture reported when the blocks were put back or saved -- and every differing slot is
+ * written to d_out (device, `cap` records) as
+ *   (block_id = d_block_ids[j], plane = p, sub_block = c, list_pos = j)
+ * in ascending (j, p, c) order.  *d_count (device, u64) receives the total, which may exceed cap; only
+ * min(count, cap) records are written.  A list position whose id lies outside [0, pool->n_blocks) was skipped by
+ * the calls that produced the digests and is never reported, whatever its slots hold.  Only n_planes, n_blocks,
+ * block_bytes and flags of `pool` are read.
+ *   d_scratch  (device) GMS_KV_VERIFY_SCRATCH_WORDS(n_sel*n_planes*k) u32 of working memory owned by the caller
+ *              (the KV calls have no manifest to keep it in); contents before and after are meaningless, and
+ *              two calls that overlap on the GPU must not share it
+ * Errors: NULL, ALIGN, ARG, RANGE, CUDA.
+ */
+typedef struct {
+    uint32_t block_id;  /* pool block, as given in the id list                        */
+    uint32_t plane;     /* layer x {K,V} plane                                        */
+    uint32_t sub_block; /* 4 KiB block inside the KV block                            */
+    uint32_t list_pos;  /* position of the block in the id list                       */
+} gms_kv_mismatch;
+#define GMS_KV_VERIFY_SCRATCH_WORDS(n_slots) (((uint64_t)(n_slots) + 2047u) / 2048u + 1u)
+int gms_kv_verify(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t n_sel, const uint64_t *d_computed,
+                  const uint64_t *d_expected, gms_kv_mismatch *d_out, uint32_t cap, uint64_t *d_count, uint32_t *d_scratch,
+                  void *stream);
 
 /*
  * Pinned, device-mapped host memory for a GMS_SRC_HOST_MAPPED image (the
@@ -456,6 +488,22 @@ int gms_service_detach(gms_service *s);
 int gms_service_reattach(gms_service *s);
 int gms_service_release_pages(gms_service *s);
 int gms_service_back_pages(gms_service *s);
+
+/*
+ * Tuning and test hooks.  The library reads the environment variables below once per process (the chunk lengths
+ * once per gms_manifest_build), and ONLY if GMS_TUNING_HOOKS=1 is set as well; without that switch none of them has
+ * any effect, so a stray variable in a serving process cannot change launch shapes or chunking.  Every setting
+ * gives bit-identical results (the test suite runs the parity checks under several of them); the defaults are what
+ * the published timings were taken with.
+ *   GMS_GEOM_RESTORE / GMS_GEOM_DIGEST / GMS_GEOM_KV   "warps,slots,CTAs-per-SM" of the restore/capture kernel, the
+ *       digest-only kernels and the KV copy kernels (defaults 9,4,1 / 16,3,1 / 8,6,1; warps 1..16, slots 3|4|6|8)
+ *   GMS_CLAIM_RESTORE / GMS_CLAIM_DIGEST               "counters,chunks-per-claim" of the work-list claims
+ *       (defaults 1,1 / 2,1; counters 1..32, chunks 1..64)
+ *   GMS_CHUNK_BLOCKS / GMS_CHUNK_BLOCKS_DIGEST         4 KiB blocks per chunk of the copy list and of the digest
+ *       list (defaults 4 / 8, fewer for small manifests; 1..32)
+ *   GMS_L2_HINTS                                       L2 eviction hints of the bulk copies, bits 0-1 loads and
+ *       2-3 stores: 0 none (default), 1 evict_first, 2 evict_last
+ */
 
 /* Launch geometry of the streaming kernels on the current device (for reporting). */
 int gms_launch_geometry(uint32_t *grid_ctas, uint32_t *warps_per_cta, uint32_t *smem_bytes);

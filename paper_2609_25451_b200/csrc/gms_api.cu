@@ -20,7 +20,8 @@ using gms::Chunk;
 struct gms_manifest {
     std::vector<gms_entry> entries;
     std::vector<uint64_t> block_base;  // n + 1 prefix sums of per-tensor block counts
-    std::vector<Chunk> chunks;
+    std::vector<Chunk> chunks;         // work list of the copying kernels (restore, capture)
+    std::vector<Chunk> digest_chunks;  // work list of the digest-only kernel: the same tensors cut into longer runs
     uint64_t image_bytes = 0, payload = 0, n_blocks = 0;
     bool host_only = false;
     bool selftest_stall = false;  // GMS_BUILD_SELFTEST_STALL
@@ -28,7 +29,7 @@ struct gms_manifest {
     int device = -1;
     // device tables (one allocation) and the recorded digests (allocated on first use)
     uint8_t *d_tables = nullptr;
-    Chunk *d_chunks = nullptr;
+    Chunk *d_chunks = nullptr, *d_digest_chunks = nullptr;
     uint64_t *d_block_base = nullptr, *d_tensor_ids = nullptr;
     uint32_t *d_seg_count = nullptr;
     unsigned int *d_counter = nullptr;
@@ -65,10 +66,10 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Cut every tensor into runs of at most `chunk_blocks` digest blocks.  Large runs first, so that
 // the dynamic claim order ends on the small ones and the last wave of warps finishes together.
-void build_chunks(gms_manifest &m, uint32_t chunk_blocks)
+void build_chunks(const gms_manifest &m, uint32_t chunk_blocks, std::vector<Chunk> &out)
 {
     const uint64_t chunk_bytes = (uint64_t)chunk_blocks * gms::kBlockBytes;
-    m.chunks.clear();
+    out.clear();
     for (size_t t = 0; t < m.entries.size(); ++t) {
         const gms_entry &e = m.entries[t];
         for (uint64_t off = 0; off < e.nbytes; off += chunk_bytes) {
@@ -79,10 +80,22 @@ void build_chunks(gms_manifest &m, uint32_t chunk_blocks)
             c.tensor = (uint32_t)t;
             c.gblock0 = (uint32_t)(m.block_base[t] + off / gms::kBlockBytes);
             c.tblock0 = (uint32_t)(off / gms::kBlockBytes);
-            m.chunks.push_back(c);
+            out.push_back(c);
         }
     }
-    std::stable_sort(m.chunks.begin(), m.chunks.end(), [](const Chunk &a, const Chunk &b) { return a.nbytes > b.nbytes; });
+    std::stable_sort(out.begin(), out.end(), [](const Chunk &a, const Chunk &b) { return a.nbytes > b.nbytes; });
+}
+
+// Tuning and test hooks read from the environment are honoured only when GMS_TUNING_HOOKS=1 is set as well, so
+// that a stray variable in a serving process changes nothing (they are listed in include/gms.h).
+long env_hook(const char *name, long lo, long hi, long fallback)
+{
+    const char *on = getenv("GMS_TUNING_HOOKS");
+    if (!on || atoi(on) != 1) return fallback;
+    const char *v = getenv(name);
+    if (!v) return fallback;
+    const long x = atol(v);
+    return x >= lo && x <= hi ? x : fallback;
 }
 
 int check_kind(const void *image, uint32_t kind)
@@ -237,7 +250,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         m->block_base[n] = acc;
 
         // ---- chunk length (needs the number of warps the restore kernel runs; a B200's if no device is asked)
-        uint32_t total_warps = 148 * 9;
+        uint32_t total_warps = 148 * 9, digest_warps = 148 * 16;
         if (!m->host_only) {
             gms::Geometry g;
             cudaError_t e = gms::get_geometry(gms::kRestore, &g);
@@ -246,23 +259,32 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
                 return cuda_fail(e);
             }
             total_warps = g.grid * g.warps;
+            if ((e = gms::get_geometry(gms::kDigest, &g)) != cudaSuccess) {
+                delete m;
+                return cuda_fail(e);
+            }
+            digest_warps = g.grid * g.warps;
             (void)cudaGetDevice(&m->device);
         }
         // Chunk length: 4 blocks (16 KiB).  Claims are made in strict list order, so short chunks keep all bytes in
         // flight within a narrow moving window of the image, which HBM rewards; shorter than 4 and the per-chunk
         // work shows.  Manifests too small to give every warp two such chunks are cut finer.
         uint32_t chunk_blocks = (uint32_t)std::min<uint64_t>(4, std::max<uint64_t>(1, (n_blocks + 2ull * total_warps - 1) / (2ull * total_warps)));
-        if (const char *v = getenv("GMS_CHUNK_BLOCKS")) {  // internal tuning / test hook
-            const long x = atol(v);
-            if (x >= 1 && x <= (long)gms::kMaxChunkBlocks) chunk_blocks = (uint32_t)x;
-        }
-        build_chunks(*m, chunk_blocks);
+        chunk_blocks = (uint32_t)env_hook("GMS_CHUNK_BLOCKS", 1, gms::kMaxChunkBlocks, chunk_blocks);
+        build_chunks(*m, chunk_blocks, m->chunks);
+        // The digest-only kernel reads twice as fast as the restore kernel moves payload and has no store side to
+        // keep narrow: it is fastest on runs of 8 blocks (32 KiB) -- 2.25 ms against 2.40 ms with 4-block chunks on
+        // a 16 GB manifest -- while the restore slows down on anything longer than 4.  So it gets a list of its own.
+        uint32_t digest_blocks = (uint32_t)std::min<uint64_t>(8, std::max<uint64_t>(1, (n_blocks + 2ull * digest_warps - 1) / (2ull * digest_warps)));
+        digest_blocks = (uint32_t)env_hook("GMS_CHUNK_BLOCKS_DIGEST", 1, gms::kMaxChunkBlocks, digest_blocks);
+        build_chunks(*m, digest_blocks, m->digest_chunks);
         m->n_segments = (uint32_t)((n_blocks + gms::kVerifySegBlocks - 1) / gms::kVerifySegBlocks);
 
         // ---- device tables
         if (!m->host_only) {
             const size_t o_chunks = 0;
-            const size_t o_base = align_up(o_chunks + m->chunks.size() * sizeof(Chunk), 256);
+            const size_t o_dchunks = align_up(o_chunks + m->chunks.size() * sizeof(Chunk), 256);
+            const size_t o_base = align_up(o_dchunks + m->digest_chunks.size() * sizeof(Chunk), 256);
             const size_t o_ids = align_up(o_base + (n + 1) * sizeof(uint64_t), 256);
             const size_t o_segcnt = align_up(o_ids + n * sizeof(uint64_t), 256);
             const size_t o_ctr = align_up(o_segcnt + (size_t)m->n_segments * sizeof(uint32_t), 256);
@@ -270,6 +292,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             const size_t total = o_status + 128;
             std::vector<uint8_t> h(total, 0);
             if (!m->chunks.empty()) memcpy(h.data() + o_chunks, m->chunks.data(), m->chunks.size() * sizeof(Chunk));
+            if (!m->digest_chunks.empty()) memcpy(h.data() + o_dchunks, m->digest_chunks.data(), m->digest_chunks.size() * sizeof(Chunk));
             memcpy(h.data() + o_base, m->block_base.data(), (n + 1) * sizeof(uint64_t));
             for (size_t t = 0; t < n; ++t) memcpy(h.data() + o_ids + t * 8, &entries[t].tensor_id, 8);
             cudaError_t e = cudaMalloc(&m->d_tables, total);
@@ -285,6 +308,7 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
                 return cuda_fail(e);
             }
             m->d_chunks = reinterpret_cast<Chunk *>(m->d_tables + o_chunks);
+            m->d_digest_chunks = reinterpret_cast<Chunk *>(m->d_tables + o_dchunks);
             m->d_block_base = reinterpret_cast<uint64_t *>(m->d_tables + o_base);
             m->d_tensor_ids = reinterpret_cast<uint64_t *>(m->d_tables + o_ids);
             m->d_seg_count = reinterpret_cast<uint32_t *>(m->d_tables + o_segcnt);
@@ -368,8 +392,8 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
                        uint64_t *d_tensor_digests, void *stream, bool capture = false, bool compare = false)
 {
     gms::StreamArgs a;
-    a.chunks = m->d_chunks;
-    a.n_chunks = (uint32_t)m->chunks.size();
+    a.chunks = store ? m->d_chunks : m->d_digest_chunks;
+    a.n_chunks = (uint32_t)(store ? m->chunks.size() : m->digest_chunks.size());
     a.image = static_cast<const uint8_t *>(image);
     a.block_digests = d_block_digests;
     a.tensor_digests = d_tensor_digests;
@@ -431,7 +455,7 @@ int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_misma
 {
     if (!m || !d_count || (cap && !d_out) || (m->n_blocks && !d_block_digests)) return GMS_ERR_NULL;
     if (m->host_only || !m->has_expected) return GMS_ERR_STATE;
-    gms::VerifyArgs a;
+    gms::VerifyArgs a = {};
     a.computed = d_block_digests;
     a.expected = m->d_expected;
     a.n_blocks = m->n_blocks;
@@ -451,7 +475,7 @@ int gms_verify(const gms_manifest *m, const uint64_t *d_block_digests, gms_misma
 static int verify_counted(const gms_manifest *m, const uint64_t *d_block_digests, gms_mismatch *d_out, uint32_t cap,
                           uint64_t *d_count, void *stream)
 {
-    gms::VerifyArgs a;
+    gms::VerifyArgs a = {};
     a.computed = d_block_digests;
     a.expected = m->d_expected;
     a.n_blocks = m->n_blocks;
@@ -517,6 +541,14 @@ int gms_last_device_status(const gms_manifest *m, void *stream, uint64_t *word)
     return (w & GMS_DEV_TIMEOUT) ? GMS_ERR_TIMEOUT : GMS_OK;
 }
 
+// A plane spans (n_blocks - 1) * block_stride + block_bytes bytes; with more than one plane, a smaller plane stride
+// would make planes share bytes, and a scatter into shared bytes has no defined result.
+static bool planes_overlap(const gms_kv_pool *pool)
+{
+    if (pool->n_planes < 2 || pool->n_blocks == 0) return false;
+    return pool->plane_stride < (uint64_t)(pool->n_blocks - 1) * pool->block_stride + pool->block_bytes;
+}
+
 static int kv_call(const gms_kv_pool *pool, const void *image, uint64_t img_plane_stride, uint64_t img_slot_stride,
                    uint32_t image_kind, const int32_t *d_block_ids, uint32_t n_sel, uint64_t *d_block_digests,
                    uint64_t *d_kv_digests, uint64_t *d_status, void *stream, bool capture)
@@ -531,6 +563,7 @@ static int kv_call(const gms_kv_pool *pool, const void *image, uint64_t img_plan
          img_plane_stride | img_slot_stride) & 15u)
         return GMS_ERR_ALIGN;
     if (pool->block_stride < pool->block_bytes && pool->n_blocks > 1) return GMS_ERR_ARG;
+    if (planes_overlap(pool)) return GMS_ERR_ARG;
     if (pool->flags & ~GMS_KV_IMAGE_BY_ID) return GMS_ERR_ARG;
     const uint64_t k = pool->block_bytes / gms::kBlockBytes;
     if ((uint64_t)n_sel * pool->n_planes * k >= 0xffffffffull) return GMS_ERR_RANGE;
@@ -587,6 +620,7 @@ int gms_kv_digest(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t 
     if (work && (!pool->base || !d_block_ids)) return GMS_ERR_NULL;
     if ((reinterpret_cast<uint64_t>(pool->base) | pool->plane_stride | pool->block_stride) & 15u) return GMS_ERR_ALIGN;
     if (pool->block_stride < pool->block_bytes && pool->n_blocks > 1) return GMS_ERR_ARG;
+    if (planes_overlap(pool)) return GMS_ERR_ARG;
     if (pool->flags & ~GMS_KV_IMAGE_BY_ID) return GMS_ERR_ARG;
     const uint64_t k = pool->block_bytes / gms::kBlockBytes;
     if ((uint64_t)n_sel * pool->n_planes * k >= 0xffffffffull) return GMS_ERR_RANGE;
@@ -604,6 +638,36 @@ int gms_kv_digest(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t 
     a.status = reinterpret_cast<unsigned long long *>(d_status);
     a.digest_only = 1u;
     GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
+    return GMS_OK;
+}
+
+int gms_kv_verify(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t n_sel, const uint64_t *d_computed,
+                  const uint64_t *d_expected, gms_kv_mismatch *d_out, uint32_t cap, uint64_t *d_count, uint32_t *d_scratch,
+                  void *stream)
+{
+    if (!pool || !d_count || (cap && !d_out)) return GMS_ERR_NULL;
+    if (pool->block_bytes == 0 || pool->block_bytes % gms::kBlockBytes) return GMS_ERR_ALIGN;
+    if (pool->block_bytes > gms::kMaxChunkBlocks * gms::kBlockBytes) return GMS_ERR_ARG;
+    if (pool->flags & ~GMS_KV_IMAGE_BY_ID) return GMS_ERR_ARG;
+    const uint64_t k = pool->block_bytes / gms::kBlockBytes;
+    const uint64_t n_slots = (uint64_t)n_sel * pool->n_planes * k;
+    if (n_slots >= 0xffffffffull) return GMS_ERR_RANGE;
+    if (n_slots && (!d_block_ids || !d_computed || !d_expected || !d_scratch)) return GMS_ERR_NULL;
+    gms::VerifyArgs a = {};
+    a.computed = d_computed;
+    a.expected = d_expected;
+    a.n_blocks = n_slots;
+    a.seg_count = d_scratch;
+    a.n_segments = (uint32_t)((n_slots + gms::kVerifySegBlocks - 1) / gms::kVerifySegBlocks);
+    a.out = d_out;
+    a.cap = cap;
+    a.count = d_count;
+    a.kv_ids = d_block_ids;
+    a.kv_slots_per_id = (uint32_t)(pool->n_planes * k);
+    a.kv_k = (uint32_t)k;
+    a.kv_pool_blocks = pool->n_blocks;
+    if (a.kv_slots_per_id == 0) a.kv_slots_per_id = 1;  // no planes: there are no slots, nothing is looked up
+    GMS_CUDA(gms::launch_verify(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
 }
 

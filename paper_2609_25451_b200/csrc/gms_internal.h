@@ -91,9 +91,14 @@ struct VerifyArgs {
     uint32_t n_tensors;
     uint32_t *seg_count;           // n_segments scratch (device): differing slots per segment
     uint32_t n_segments;
-    void *out;                     // gms_mismatch[cap]
+    void *out;                     // gms_mismatch[cap] (gms_kv_mismatch[cap] in KV mode)
     uint32_t cap;
     uint64_t *count;
+    // KV mode (gms_kv_verify): slots are [list position][plane][sub-block]; 0 slots per id = manifest mode
+    const int32_t *kv_ids;
+    uint32_t kv_slots_per_id;      // n_planes * (block_bytes / 4096)
+    uint32_t kv_k;                 // block_bytes / 4096
+    uint32_t kv_pool_blocks;       // ids outside [0, kv_pool_blocks) are never reported
 };
 constexpr uint32_t kVerifySegShift = 11;
 constexpr uint32_t kVerifySegBlocks = 1u << kVerifySegShift;  // digest slots compared by one CTA (one counter each)

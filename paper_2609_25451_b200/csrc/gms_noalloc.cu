@@ -78,7 +78,7 @@ extern "C" int gms_verify_flat_noalloc(const uint64_t *d_computed, const uint64_
     if ((e = cudaGetLastError()) != cudaSuccess) return gms::report_cuda_error(e);
     gms::count_launches(1);
 
-    gms::VerifyArgs a;
+    gms::VerifyArgs a = {};
     a.computed = d_computed;
     a.expected = d_expected;
     a.n_blocks = n_blocks;

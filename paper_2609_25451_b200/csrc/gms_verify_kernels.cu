@@ -24,17 +24,52 @@ struct Mismatch {
     uint64_t tensor_id, block;
 };
 
-__device__ __forceinline__ uint32_t diff_mask(const uint64_t *c, const uint64_t *x, uint64_t first, uint64_t n)
+// Whether a differing slot counts.  Manifest mode: always.  KV mode (gms_kv_verify): only if the slot belongs to a
+// list position whose block id lies inside the pool -- an id outside it was skipped by the call that produced the
+// digests and is never reported.
+template <bool kKv>
+__device__ __forceinline__ bool counts(const VerifyArgs &a, uint64_t g)
+{
+    if (!kKv) return true;
+    const int32_t id = a.kv_ids[g / a.kv_slots_per_id];
+    return id >= 0 && (uint32_t)id < a.kv_pool_blocks;
+}
+
+template <bool kKv>
+__device__ __forceinline__ uint32_t diff_mask(const VerifyArgs &a, uint64_t first)
 {
     uint32_t mask = 0;
 #pragma unroll
     for (uint32_t k = 0; k < kPerThread; ++k) {
         const uint64_t g = first + k;
-        if (g < n && c[g] != x[g]) mask |= 1u << k;
+        if (g < a.n_blocks && a.computed[g] != a.expected[g] && counts<kKv>(a, g)) mask |= 1u << k;
     }
     return mask;
 }
 
+// One output record for differing slot g.  Manifest mode: (tensor_id, block inside the tensor), found by binary
+// search of the block-base table.  KV mode: slots are laid out [list position j][plane][4 KiB sub-block], and the
+// record is (block id, plane, sub-block, j).
+template <bool kKv>
+__device__ __forceinline__ void write_record(const VerifyArgs &a, uint64_t rank, uint64_t g)
+{
+    if (kKv) {
+        const uint32_t j = (uint32_t)(g / a.kv_slots_per_id), r = (uint32_t)(g % a.kv_slots_per_id);
+        static_cast<uint4 *>(a.out)[rank] = make_uint4((uint32_t)a.kv_ids[j], r / a.kv_k, r % a.kv_k, j);
+        return;
+    }
+    // entry t with block_base[t] <= g < block_base[t+1]; empty tensors share a base and are skipped
+    uint32_t lo = 0, hi = a.n_tensors;
+    while (hi - lo > 1) {
+        const uint32_t mid = lo + (hi - lo) / 2;
+        if (a.block_base[mid] <= g) lo = mid; else hi = mid;
+    }
+    Mismatch *out = static_cast<Mismatch *>(a.out);
+    out[rank].tensor_id = a.tensor_ids[lo];
+    out[rank].block = g - a.block_base[lo];
+}
+
+template <bool kKv>
 __global__ void __launch_bounds__(kThreads) gms_verify_count_kernel(VerifyArgs a)
 {
     asm volatile("griddepcontrol.launch_dependents;");  // the emit kernel may be scheduled; it waits for our counts
@@ -51,10 +86,10 @@ __global__ void __launch_bounds__(kThreads) gms_verify_count_kernel(VerifyArgs a
         if (vec && g + 1 < a.n_blocks) {
             const ulonglong2 p = *reinterpret_cast<const ulonglong2 *>(a.computed + g);
             const ulonglong2 q = *reinterpret_cast<const ulonglong2 *>(a.expected + g);
-            c += (p.x != q.x) + (p.y != q.y);
+            c += (p.x != q.x && counts<kKv>(a, g)) + (p.y != q.y && counts<kKv>(a, g + 1));
         } else {  // arrays that are only 8-byte aligned, and the odd last slot
-            if (g < a.n_blocks) c += a.computed[g] != a.expected[g];
-            if (g + 1 < a.n_blocks) c += a.computed[g + 1] != a.expected[g + 1];
+            if (g < a.n_blocks) c += a.computed[g] != a.expected[g] && counts<kKv>(a, g);
+            if (g + 1 < a.n_blocks) c += a.computed[g + 1] != a.expected[g + 1] && counts<kKv>(a, g + 1);
         }
     }
     c = __reduce_add_sync(0xffffffffu, c);
@@ -70,6 +105,7 @@ __global__ void __launch_bounds__(kThreads) gms_verify_count_kernel(VerifyArgs a
 // Ordered emit.  CTA k owns segment k.  Its offset in the output is the sum of the counts of segments 0..k-1,
 // which it adds up itself (at most a few thousand 32-bit words, read by 256 threads); segments without
 // differences return at once, except the last one, which also publishes the total.
+template <bool kKv>
 __global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
 {
     asm volatile("griddepcontrol.launch_dependents;");
@@ -95,7 +131,7 @@ __global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
     if (last && threadIdx.x == 0) *a.count = before + own;
     if (own == 0) return;
     const uint64_t first = (uint64_t)blockIdx.x * kVerifySegBlocks + (uint64_t)threadIdx.x * kPerThread;
-    const uint32_t mask = diff_mask(a.computed, a.expected, first, a.n_blocks);
+    const uint32_t mask = diff_mask<kKv>(a, first);
     const uint32_t mine = __popc(mask);
     uint32_t incl = mine;
 #pragma unroll
@@ -108,20 +144,9 @@ __global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
     uint64_t rank = before + incl - mine;
     for (uint32_t w = 0; w < warp; ++w) rank += warp_sum[w];
     if (!mask) return;
-    Mismatch *out = static_cast<Mismatch *>(a.out);
     for (uint32_t k = 0; k < kPerThread; ++k) {
         if (!(mask & (1u << k))) continue;
-        if (rank < a.cap) {
-            const uint64_t g = first + k;
-            // entry t with block_base[t] <= g < block_base[t+1]; empty tensors share a base and are skipped
-            uint32_t lo = 0, hi = a.n_tensors;
-            while (hi - lo > 1) {
-                const uint32_t mid = lo + (hi - lo) / 2;
-                if (a.block_base[mid] <= g) lo = mid; else hi = mid;
-            }
-            out[rank].tensor_id = a.tensor_ids[lo];
-            out[rank].block = g - a.block_base[lo];
-        }
+        if (rank < a.cap) write_record<kKv>(a, rank, first + k);
         ++rank;
     }
 }
@@ -129,6 +154,7 @@ __global__ void __launch_bounds__(kThreads) gms_verify_emit_kernel(VerifyArgs a)
 // Small inputs (a few thousand digest slots): the three passes in one CTA, one launch.
 constexpr uint32_t kSmallThreads = 1024;
 constexpr uint64_t kSmallBlocks = 16384;
+template <bool kKv>
 __global__ void __launch_bounds__(kSmallThreads) gms_verify_small_kernel(VerifyArgs a)
 {
     __shared__ uint32_t warp_sum[kSmallThreads / 32];
@@ -137,7 +163,7 @@ __global__ void __launch_bounds__(kSmallThreads) gms_verify_small_kernel(VerifyA
     const uint64_t per = (a.n_blocks + kSmallThreads - 1) / kSmallThreads;  // consecutive slots per thread
     const uint64_t lo = (uint64_t)threadIdx.x * per, hi = lo + per < a.n_blocks ? lo + per : a.n_blocks;
     uint32_t mine = 0;
-    for (uint64_t g = lo; g < hi; ++g) mine += a.computed[g] != a.expected[g];
+    for (uint64_t g = lo; g < hi; ++g) mine += a.computed[g] != a.expected[g] && counts<kKv>(a, g);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t incl = mine;
 #pragma unroll
@@ -154,18 +180,9 @@ __global__ void __launch_bounds__(kSmallThreads) gms_verify_small_kernel(VerifyA
     }
     if (threadIdx.x == 0) *a.count = total;
     if (!mine) return;
-    Mismatch *out = static_cast<Mismatch *>(a.out);
     for (uint64_t g = lo; g < hi; ++g) {
-        if (a.computed[g] == a.expected[g]) continue;
-        if (rank < a.cap) {
-            uint32_t l = 0, h = a.n_tensors;
-            while (h - l > 1) {
-                const uint32_t mid = l + (h - l) / 2;
-                if (a.block_base[mid] <= g) l = mid; else h = mid;
-            }
-            out[rank].tensor_id = a.tensor_ids[l];
-            out[rank].block = g - a.block_base[l];
-        }
+        if (a.computed[g] == a.expected[g] || !counts<kKv>(a, g)) continue;
+        if (rank < a.cap) write_record<kKv>(a, rank, g);
         ++rank;
     }
 }
@@ -200,18 +217,23 @@ cudaError_t launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, cudaStream_t
 cudaError_t launch_verify_counted(const VerifyArgs &a, cudaStream_t s)
 {
     count_launches(1);
-    return launch_pdl(gms_verify_emit_kernel, dim3(a.n_segments ? a.n_segments : 1), dim3(kThreads), s, a);
+    const dim3 grid(a.n_segments ? a.n_segments : 1);
+    return a.kv_slots_per_id ? launch_pdl(gms_verify_emit_kernel<true>, grid, dim3(kThreads), s, a)
+                             : launch_pdl(gms_verify_emit_kernel<false>, grid, dim3(kThreads), s, a);
 }
 
 cudaError_t launch_verify(const VerifyArgs &a, cudaStream_t s)
 {
+    const bool kv = a.kv_slots_per_id != 0;
     if (a.n_segments == 0) return launch_verify_counted(a, s);  // no digest slots at all: count = 0
     if (a.n_blocks <= kSmallBlocks) {
         count_launches(1);
-        return launch_pdl(gms_verify_small_kernel, dim3(1), dim3(kSmallThreads), s, a);
+        return kv ? launch_pdl(gms_verify_small_kernel<true>, dim3(1), dim3(kSmallThreads), s, a)
+                  : launch_pdl(gms_verify_small_kernel<false>, dim3(1), dim3(kSmallThreads), s, a);
     }
     count_launches(1);
-    cudaError_t e = launch_pdl(gms_verify_count_kernel, dim3(a.n_segments), dim3(kThreads), s, a);
+    cudaError_t e = kv ? launch_pdl(gms_verify_count_kernel<true>, dim3(a.n_segments), dim3(kThreads), s, a)
+                       : launch_pdl(gms_verify_count_kernel<false>, dim3(a.n_segments), dim3(kThreads), s, a);
     if (e) return e;
     return launch_verify_counted(a, s);
 }

@@ -29,11 +29,12 @@ DEV_TIMEOUT = 1  # bit of the device status word
 # numpy view of gms_entry / gms_mismatch (32 and 16 bytes)
 ENTRY_DTYPE = np.dtype([("tensor_id", "<u8"), ("src_offset", "<u8"), ("dst", "<u8"), ("nbytes", "<u8")])
 MISMATCH_DTYPE = np.dtype([("tensor_id", "<u8"), ("block", "<u8")])
+KV_MISMATCH_DTYPE = np.dtype([("block_id", "<u4"), ("plane", "<u4"), ("sub_block", "<u4"), ("list_pos", "<u4")])
 
 EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
-    "gms_verify", "gms_digest_verify", "gms_restore_verify", "gms_verify_tensors", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_kv_digest", "gms_host_image_alloc", "gms_host_image_free",
+    "gms_verify", "gms_digest_verify", "gms_restore_verify", "gms_verify_tensors", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_kv_digest", "gms_kv_verify", "gms_host_image_alloc", "gms_host_image_free",
     "gms_pipe_create", "gms_pipe_destroy", "gms_restore_fd", "gms_stage_create", "gms_stage_destroy", "gms_restore_staged",
     "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
     "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
@@ -92,6 +93,7 @@ def lib():
             "gms_kv_restore": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
             "gms_kv_capture": (i, [C.POINTER(KvPool), p, u64, u64, u32, p, u32, p, p, p, p]),
             "gms_kv_digest": (i, [C.POINTER(KvPool), p, u32, p, p, p, p]),
+            "gms_kv_verify": (i, [C.POINTER(KvPool), p, u32, p, p, p, u32, p, p, p]),
             "gms_host_image_alloc": (i, [u64, pp, pp]),
             "gms_host_image_free": (i, [p]),
             "gms_pipe_create": (i, [u32, u64, u32, pp]),
@@ -270,6 +272,17 @@ def gms_kv_capture(pool: KvPool, image, img_plane_stride: int, img_slot_stride: 
 def gms_kv_digest(pool: KvPool, d_block_ids, n_sel: int, d_block_digests, d_kv_digests, d_status, stream=None):
     _check(lib().gms_kv_digest(C.byref(pool), _dev(d_block_ids), n_sel, _dev(d_block_digests), _dev(d_kv_digests),
                                _dev(d_status), _stream(stream)), "gms_kv_digest")
+
+
+def kv_verify_scratch_words(n_slots: int) -> int:
+    """GMS_KV_VERIFY_SCRATCH_WORDS of include/gms.h: u32 words of caller-owned working memory for gms_kv_verify."""
+    return (int(n_slots) + 2047) // 2048 + 1
+
+
+def gms_kv_verify(pool: KvPool, d_block_ids, n_sel: int, d_computed, d_expected, d_out, cap: int, d_count, d_scratch,
+                  stream=None):
+    _check(lib().gms_kv_verify(C.byref(pool), _dev(d_block_ids), n_sel, _dev(d_computed), _dev(d_expected), _dev(d_out), cap,
+                               _dev(d_count), _dev(d_scratch), _stream(stream)), "gms_kv_verify")
 
 
 def gms_host_image_alloc(nbytes: int):

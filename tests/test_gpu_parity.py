@@ -137,12 +137,23 @@ def test_results_do_not_depend_on_entry_order_or_chunking(oracle, monkeypatch):
     assert {int(r["tensor_id"]): int(td2[t]) for t, r in enumerate(w2.rows)} == by_id
     d2.close()
     # different internal chunk length: every output bit-identical
-    for blocks in ("1", "5", "32"):
+    monkeypatch.setenv("GMS_TUNING_HOOKS", "1")
+    for blocks, digest_blocks in (("1", "32"), ("5", "3"), ("32", "1")):
         monkeypatch.setenv("GMS_CHUNK_BLOCKS", blocks)
+        monkeypatch.setenv("GMS_CHUNK_BLOCKS_DIGEST", digest_blocks)
         d3 = DeviceWorkload(w, image)
+        assert gms.gms_manifest_chunk(d3.m, 0)[2] == min(int(blocks) * 4096, int(w.rows["nbytes"].max()))
         bd3, td3 = d3.restore()
         assert np.array_equal(bd3, bd) and np.array_equal(td3, td) and np.array_equal(d3.slab_host(), slab)
+        bd4, td4 = d3.digest()
+        assert np.array_equal(bd4, bd) and np.array_equal(td4, td)
         d3.close()
+    # without the master switch the hooks are ignored
+    monkeypatch.delenv("GMS_TUNING_HOOKS")
+    monkeypatch.setenv("GMS_CHUNK_BLOCKS", "1")
+    d4 = DeviceWorkload(w, image)
+    assert gms.gms_manifest_chunk(d4.m, 0)[2] > 4096
+    d4.close()
 
 
 @pytest.mark.parametrize("scale", [1, 8])  # 8.7 K blocks: single-CTA verify; 70 K blocks: count / scan / emit

@@ -25,8 +25,9 @@ SHAPES = [
     {"GMS_GEOM_RESTORE": "12,4,1", "GMS_GEOM_DIGEST": "12,4,1", "GMS_GEOM_KV": "12,4,1", "GMS_CHUNK_BLOCKS": "1"},
     {"GMS_GEOM_RESTORE": "6,8,1", "GMS_GEOM_DIGEST": "6,8,1", "GMS_GEOM_KV": "6,8,1", "GMS_CHUNK_BLOCKS": "32"},
     {"GMS_GEOM_RESTORE": "6,4,2", "GMS_GEOM_DIGEST": "8,3,2", "GMS_GEOM_KV": "4,6,2", "GMS_CLAIM_RESTORE": "8,3",
-     "GMS_CLAIM_DIGEST": "1,1", "GMS_CHUNK_BLOCKS": "7"},
-    {"GMS_GEOM_RESTORE": "16,3,1", "GMS_CLAIM_RESTORE": "32,2", "GMS_CLAIM_DIGEST": "32,64", "GMS_L2_HINTS": "5"},
+     "GMS_CLAIM_DIGEST": "1,1", "GMS_CHUNK_BLOCKS": "7", "GMS_CHUNK_BLOCKS_DIGEST": "2"},
+    {"GMS_GEOM_RESTORE": "16,3,1", "GMS_CLAIM_RESTORE": "32,2", "GMS_CLAIM_DIGEST": "32,64", "GMS_L2_HINTS": "5",
+     "GMS_CHUNK_BLOCKS_DIGEST": "32"},
 ]
 
 
@@ -34,6 +35,7 @@ SHAPES = [
 def test_parity_in_other_launch_shapes(env):
     full = dict(os.environ)
     full.update(env)
+    full["GMS_TUNING_HOOKS"] = "1"  # the library ignores the shape hooks without it
     r = subprocess.run([sys.executable, os.path.join(HERE, "geometry_check.py")], env=full, capture_output=True, text=True,
                        timeout=600)
     assert r.returncode == 0 and r.stdout.strip().startswith("OK"), r.stdout[-2000:] + r.stderr[-4000:]

@@ -169,6 +169,20 @@ def test_kv_argument_checks_need_no_gpu():
     assert call(pool, kind=7) == gms.ERR_KIND
     assert call(pool, iss=32760) == gms.ERR_ALIGN
     assert gms.lib().gms_kv_restore(None, None, 0, 0, 0, None, 0, None, None, st, None) == gms.ERR_NULL
+    # planes that would share bytes: a plane spans (n_blocks - 1) * block_stride + block_bytes
+    span = 7 * 32768 + 32768
+    tight = gms.KvPool(base=FAKE_BASE, plane_stride=span - 16, block_stride=32768, n_planes=2, n_blocks=8, block_bytes=32768)
+    assert call(tight) == gms.ERR_ARG
+    assert gms.lib().gms_kv_digest(ctypes.byref(tight), ctypes.c_void_p(FAKE_BASE), 4, None, None, st, None) == gms.ERR_ARG
+    one_plane = gms.KvPool(base=FAKE_BASE, plane_stride=0, block_stride=32768, n_planes=1, n_blocks=8, block_bytes=32768)
+    assert call(one_plane, kind=7) == gms.ERR_KIND  # a single plane has no neighbour to overlap: the check is passed
+    # gms_kv_verify: host-side checks
+    kvv = lambda p, n_sel=4, ids=FAKE_BASE, cap=4: gms.lib().gms_kv_verify(
+        ctypes.byref(p), ctypes.c_void_p(ids), n_sel, ctypes.c_void_p(FAKE_BASE), ctypes.c_void_p(FAKE_BASE),
+        ctypes.c_void_p(FAKE_BASE), cap, st, None, None)
+    assert kvv(bad) == gms.ERR_ALIGN and kvv(big) == gms.ERR_ARG
+    assert kvv(pool) == gms.ERR_NULL  # slots to compare but no scratch
+    assert gms.kv_verify_scratch_words(0) == 1 and gms.kv_verify_scratch_words(2048) == 2 and gms.kv_verify_scratch_words(2049) == 3
 
 
 def test_workload_recipes_have_the_stated_sizes():
