@@ -46,11 +46,14 @@ METRIC = "restore+digest GB/s"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 DATASHEET_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum per payload byte, taken from the ncu captures summarised under
-# profiles/ (small cases of the same kernels; the traffic is proportional to the payload).  Not measured by this run.
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"restore_verify": 2.000, "restore": 2.000, "digest_verify": 1.004, "digest": 1.004,
-                                   "kv_restore": 1.993, "capture": 1.983}
-NCU_TRAFFIC_SOURCE = "profiles/ (ncu dram__bytes of a small case of the same kernel x payload; not measured in this run)"
+# dram__bytes_read.sum + dram__bytes_write.sum per payload byte, from the ncu captures summarised under profiles/
+# (small cases of the same kernels: a 1 GB manifest of the 8B structure, a 6 GB KV pool).  Traffic grows in
+# proportion to the payload, except that the write side of a small case is short by what L2 still holds when the
+# kernel ends (about 50 MB); the figures are used as they were measured.  Not measured by this run.
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"restore_verify": 1.955, "restore": 1.955, "digest_verify": 1.008, "digest": 1.008,
+                                   "kv_restore": 1.919, "capture": None}
+NCU_TRAFFIC_SOURCE = ("profiles/stream_kernels_llama3-8b-shrink4_ncu_full.md, profiles/kv_stream_kernels_6GB_pool_ncu_full.md: "
+                      "ncu dram__bytes of a small case of the same kernel, per payload byte, x this payload (not measured in this run)")
 CONFIG_ORDER = ["tiny", "8b", "kv", "mixed", "host70b"]
 
 
@@ -73,6 +76,7 @@ def parse_args():
     ap.add_argument("--pipe-buffers", type=int, default=4)
     ap.add_argument("--pipe-mib", type=int, default=256)
     ap.add_argument("--pipe-readers", type=int, default=16)
+    ap.add_argument("--direct-io", action="store_true", help="file: O_DIRECT reads where the file system takes them (cold files on fast storage)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -965,6 +969,7 @@ def run_file(args, torch, gms, W, dev, index, want_cpu=True):
         link_gbs = h2d_yardstick(torch, torch.from_numpy(arr), bench.image[:buf_bytes], reps=5)
         gms.gms_host_image_free(hptr)
         pipe = gms.gms_pipe_create(n_buf, buf_bytes, n_readers)
+        gms.gms_pipe_direct_io(pipe, args.direct_io)
         gms.gms_restore_fd(bench.m, pipe, fd, 0, bench.bd, bench.td)
         steps = max(1, min(args.steps, 5))
         sampler = ClockSampler(index)

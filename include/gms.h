@@ -373,9 +373,15 @@ int gms_host_image_free(void *host_ptr);
  * gms_pipe_* / gms_restore_fd -- Section 4, GMS paragraph: with a cold service, a fresh writer
  * fills the model state in from storage while the process is being restored; Section 3.1 prices it
  * at S / B_eff.  The image is read from a file descriptor, never resident as a whole: a ring of
- * `n_buffers` pinned, device-mapped buffers of `buffer_bytes` each (>= 1 MiB, multiple of 4096) is
- * filled by `n_readers` threads with pread(), and each filled buffer is consumed by the restore
- * kernel (which reads it across the host link, scatters and digests) while the next one is read.
+ * `n_buffers` pinned buffers of `buffer_bytes` each (>= 1 MiB, multiple of 4096) is filled by
+ * `n_readers` threads with pread(), with a read-ahead hint for the window after (and, after
+ * gms_pipe_direct_io(p, 1), bypassing the page cache with O_DIRECT where the file system allows it:
+ * right for a cold snapshot on fast storage, wrong for a file the page cache already holds, so it is
+ * off unless asked for), and each filled buffer is moved by the
+ * copy engine into one of two device buffers of the same size (allocated by gms_pipe_create) and
+ * scattered + digested from there by the restore kernel while the next one is read.  If the device
+ * buffers cannot be allocated the pipe still works: the kernel then reads the pinned buffers across
+ * the host link itself, which reaches about 93 % of what the copy engine does.
  * The first gms_restore_fd (or gms_restore_staged) on a manifest builds and uploads a copy of its work list
  * sorted by source offset: that call allocates device memory and synchronises, so it must not be made
  * while a stream capture is in progress.
@@ -391,8 +397,11 @@ typedef struct {
     double wait_read_seconds;  /* host time spent waiting for readers (storage-bound share) */
     double wait_gpu_seconds;   /* host time spent waiting for a buffer to be released       */
     double total_seconds;      /* wall time of the call                                     */
+    uint32_t direct_io;        /* 1: the file system accepted O_DIRECT reads                */
+    uint32_t copy_engine;      /* 1: windows went pinned buffer -> copy engine -> device    */
 } gms_pipe_stats;
 int gms_pipe_create(uint32_t n_buffers, uint64_t buffer_bytes, uint32_t n_readers, gms_pipe **out);
+int gms_pipe_direct_io(gms_pipe *p, int enable);
 int gms_pipe_destroy(gms_pipe *p);
 int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_offset, uint64_t *d_block_digests,
                    uint64_t *d_tensor_digests, void *stream, gms_pipe_stats *stats);

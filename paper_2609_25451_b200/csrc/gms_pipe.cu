@@ -3,11 +3,14 @@
 // Section 4 (GMS paragraph) has a fresh writer fill a cold service from storage while the process
 // itself is being restored; Section 3.1 prices that at S / B_eff and Section 3.3 notes that restoring
 // the runtime state leaves storage bandwidth unused.  This file is that leg: the snapshot
-// image is never resident as a whole.  A small ring of pinned, device-mapped buffers is filled by a
-// pool of reader threads (pread), and as soon as a buffer holds a window of the image the restore
-// kernel is launched on the chunks whose sources lie in that window, reading the pinned buffer
-// across the host link and scattering + digesting as usual.  Reading window k+1 overlaps the kernel
-// of window k; a buffer is refilled only after the kernel that read it has finished (CUDA event).
+// image is never resident as a whole.  A small ring of pinned buffers is filled by a pool of reader
+// threads (pread; O_DIRECT where the file system takes it, the page cache otherwise), each filled
+// buffer is moved by the copy engine (cudaMemcpyAsync on an internal stream) into one of two device
+// buffers, and the restore kernel is launched on the chunks whose sources lie in that window, reading
+// device memory and scattering + digesting as usual.  Reading window k+1 overlaps the copy and the
+// kernel of window k; a pinned buffer is refilled once its copy has completed, a device buffer once
+// the kernel that read it has (CUDA events).  If the device buffers cannot be had, the kernel reads the
+// pinned buffers across the host link instead (about 7 % slower on the link).
 // All waiting is on the host (condition variables, cudaEventSynchronize); no kernel waits for a flag.
 #include <condition_variable>
 #include <cerrno>
@@ -18,6 +21,8 @@
 #include <thread>
 #include <vector>
 
+#include <atomic>
+#include <fcntl.h>
 #include <unistd.h>
 
 #include "../../include/gms.h"
@@ -92,7 +97,14 @@ struct gms_pipe {
     uint64_t buffer_bytes = 0;
     std::vector<void *> host;    // pinned buffers
     std::vector<void *> dview;   // their device-side addresses
-    std::vector<cudaEvent_t> done;
+    std::vector<cudaEvent_t> done;  // the last reader of pinned buffer b (copy, or kernel when there is no device ring) is finished
+    // device ring fed by the copy engine (empty: kernels read the pinned buffers themselves)
+    std::vector<void *> dev;
+    std::vector<cudaEvent_t> copied;    // device buffer d holds its window (recorded on the copy stream)
+    std::vector<cudaEvent_t> consumed;  // the kernel that read device buffer d has finished (caller's stream)
+    cudaStream_t copy_stream = nullptr;
+    uint64_t dev_uses = 0;              // windows pushed through the device ring so far (across calls)
+    bool direct_io = false;             // gms_pipe_direct_io: read with O_DIRECT where the file system allows it
     ReaderPool *pool = nullptr;
     std::mutex busy;             // one restore at a time per pipe
 };
@@ -229,9 +241,33 @@ int gms_pipe_create(uint32_t n_buffers, uint64_t buffer_bytes, uint32_t n_reader
         p->pool = new (std::nothrow) ReaderPool(n_readers);
         if (!p->pool) rc = GMS_ERR_NOMEM;
     }
+    if (rc == GMS_OK) {  // two device buffers for the copy engine to fill; without them the mapped path is used
+        cudaError_t e = cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking);
+        for (uint32_t d = 0; d < 2 && e == cudaSuccess; ++d) {
+            void *buf = nullptr;
+            cudaEvent_t a = nullptr, c = nullptr;
+            e = cudaMalloc(&buf, buffer_bytes);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&a, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c, cudaEventDisableTiming);
+            if (buf) p->dev.push_back(buf);
+            if (a) p->copied.push_back(a);
+            if (c) p->consumed.push_back(c);
+        }
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            for (void *buf : p->dev) cudaFree(buf);
+            for (cudaEvent_t ev : p->copied) cudaEventDestroy(ev);
+            for (cudaEvent_t ev : p->consumed) cudaEventDestroy(ev);
+            p->dev.clear();
+            p->copied.clear();
+            p->consumed.clear();
+            if (e != cudaErrorMemoryAllocation) rc = gms::report_cuda_error(e);
+        }
+    }
     if (rc != GMS_OK) {
         for (void *h : p->host) cudaFreeHost(h);
         for (cudaEvent_t ev : p->done) cudaEventDestroy(ev);
+        if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
         delete p->pool;
         delete p;
         return rc;
@@ -240,11 +276,27 @@ int gms_pipe_create(uint32_t n_buffers, uint64_t buffer_bytes, uint32_t n_reader
     return GMS_OK;
 }
 
+int gms_pipe_direct_io(gms_pipe *p, int enable)
+{
+    if (!p) return GMS_ERR_NULL;
+    std::lock_guard<std::mutex> one(p->busy);
+    p->direct_io = enable != 0;
+    return GMS_OK;
+}
+
 int gms_pipe_destroy(gms_pipe *p)
 {
     if (!p) return GMS_OK;
     delete p->pool;  // joins the readers
     int rc = GMS_OK;
+    if (p->copy_stream && cudaStreamSynchronize(p->copy_stream) != cudaSuccess) rc = GMS_ERR_CUDA;
+    for (cudaEvent_t ev : p->consumed)
+        if (cudaEventSynchronize(ev) != cudaSuccess) rc = GMS_ERR_CUDA;
+    for (void *buf : p->dev)
+        if (cudaFree(buf) != cudaSuccess) rc = GMS_ERR_CUDA;
+    for (cudaEvent_t ev : p->copied) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : p->consumed) cudaEventDestroy(ev);
+    if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
     for (cudaEvent_t ev : p->done)
         if (cudaEventDestroy(ev) != cudaSuccess) rc = GMS_ERR_CUDA;
     for (void *h : p->host)
@@ -261,7 +313,8 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
     std::lock_guard<std::mutex> one(p->busy);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     std::vector<gms::SrcWindow> windows;
-    int rc = gms::manifest_src_windows(m, p->buffer_bytes, &windows);
+    // a window is read from the 4 KiB boundary below its first byte (so that direct reads stay aligned): leave room
+    int rc = gms::manifest_src_windows(m, p->buffer_bytes - 4096, &windows);
     if (rc != GMS_OK) return rc;
     const double t_start = now_s();
     gms_pipe_stats st = {};
@@ -276,6 +329,19 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
     const uint32_t n_readers = p->pool->size();
     size_t next_read = 0, next_launch = 0;
     int io_error = 0;
+    const bool staged = !p->dev.empty();
+    // On request (gms_pipe_direct_io): a second descriptor on the same file that bypasses the page cache, where the
+    // file system allows it (where it does not, the open or the first read fails and the ordinary descriptor is used).
+    // Direct reads need 4 KiB-aligned file offsets, addresses and lengths, so every window is read from the 4 KiB
+    // boundary below its first byte and used from `shift` bytes into its buffer (the kernel's sources must stay
+    // 16-byte aligned, which they do when file_offset is a multiple of 16; otherwise nothing is shifted and only
+    // slices that happen to be aligned go direct).
+    char proc_path[64];
+    snprintf(proc_path, sizeof proc_path, "/proc/self/fd/%d", fd);
+    const int dfd = p->direct_io ? open(proc_path, O_RDONLY | O_DIRECT | O_CLOEXEC) : -1;
+    std::atomic<bool> direct_ok{dfd >= 0};
+    const bool shifted = dfd >= 0 && (file_offset & 15u) == 0;
+    std::vector<uint32_t> shifts(windows.size(), 0);
     while (rc == GMS_OK && next_launch < windows.size()) {
         // start reads as far ahead as the ring allows
         while (next_read < windows.size() && next_read < next_launch + p->n_buffers) {
@@ -292,18 +358,39 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
             const gms::SrcWindow &w = windows[next_read];
             WindowReads &wr = reads[next_read];
             const uint64_t len = w.src_hi - w.src_lo;
+            if (next_read + 1 < windows.size())  // tell the kernel which bytes come next (a hint; errors do not matter)
+                (void)posix_fadvise(fd, (off_t)(file_offset + windows[next_read + 1].src_lo),
+                                    (off_t)(windows[next_read + 1].src_hi - windows[next_read + 1].src_lo), POSIX_FADV_WILLNEED);
+            const uint64_t shift = shifted ? ((file_offset + w.src_lo) & 4095u) : 0;
+            shifts[next_read] = (uint32_t)shift;
+            const uint64_t span = len + shift;  // bytes read into the buffer, from its start
             // slices are multiples of 1 MiB so that readers do not share pages
-            uint64_t slice = (len + n_readers - 1) / n_readers;
+            uint64_t slice = (span + n_readers - 1) / n_readers;
             slice = (slice + (1u << 20) - 1) & ~((uint64_t)(1u << 20) - 1);
-            const uint32_t n_slices = (uint32_t)((len + slice - 1) / slice);
+            const uint32_t n_slices = (uint32_t)((span + slice - 1) / slice);
             wr.pending = n_slices;
             uint8_t *base = static_cast<uint8_t *>(p->host[b]);
             for (uint32_t k = 0; k < n_slices; ++k) {
-                const uint64_t lo = (uint64_t)k * slice, n = std::min<uint64_t>(slice, len - lo);
-                const uint64_t foff = file_offset + w.src_lo + lo;
-                p->pool->submit([fd, base, lo, n, foff, &wr] {
+                const uint64_t lo = (uint64_t)k * slice, n = std::min<uint64_t>(slice, span - lo);
+                const uint64_t foff = file_offset + w.src_lo - shift + lo;
+                p->pool->submit([fd, dfd, &direct_ok, base, lo, n, foff, &wr] {
                     uint64_t got = 0;
                     int err = 0;
+                    // the 4 KiB-aligned body of the slice through the direct descriptor, if it still works
+                    const uint64_t body = n & ~(uint64_t)4095;
+                    if (body && direct_ok.load(std::memory_order_relaxed) && (foff & 4095u) == 0 &&
+                        (reinterpret_cast<uint64_t>(base + lo) & 4095u) == 0) {
+                        while (got < body) {
+                            const ssize_t r = pread(dfd, base + lo + got, body - got, (off_t)(foff + got));
+                            if (r < 0 && errno == EINTR) continue;
+                            if (r <= 0 || (r & 4095)) {  // refused, short or ragged: the ordinary descriptor takes over
+                                if (r < 0) direct_ok.store(false, std::memory_order_relaxed);
+                                if (r > 0) got += (uint64_t)r;
+                                break;
+                            }
+                            got += (uint64_t)r;
+                        }
+                    }
                     while (got < n) {
                         const ssize_t r = pread(fd, base + lo + got, n - got, (off_t)(foff + got));
                         if (r < 0) {
@@ -339,11 +426,33 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
             }
         }
         const uint32_t b = (uint32_t)(next_launch % p->n_buffers);
-        rc = gms::manifest_launch_window(m, windows[next_launch], p->dview[b], next_launch == 0, d_block_digests,
-                                         d_tensor_digests, s);
-        if (rc == GMS_OK) {
-            cudaError_t e = cudaEventRecord(p->done[b], s);
-            if (e != cudaSuccess) rc = gms::report_cuda_error(e);
+        if (staged) {
+            // copy engine: pinned buffer b -> device buffer d (once the kernel that last read d is done), then the
+            // kernel on the caller's stream reads d; the pinned buffer is free again when the copy has completed
+            const uint32_t d = (uint32_t)(p->dev_uses % p->dev.size());
+            const gms::SrcWindow &w = windows[next_launch];
+            cudaError_t e = cudaSuccess;
+            if (p->dev_uses >= p->dev.size()) e = cudaStreamWaitEvent(p->copy_stream, p->consumed[d], 0);
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync(p->dev[d], static_cast<const uint8_t *>(p->host[b]) + shifts[next_launch], w.src_hi - w.src_lo,
+                                    cudaMemcpyHostToDevice, p->copy_stream);
+            if (e == cudaSuccess) e = cudaEventRecord(p->copied[d], p->copy_stream);
+            if (e == cudaSuccess) e = cudaEventRecord(p->done[b], p->copy_stream);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(s, p->copied[d], 0);
+            if (e != cudaSuccess) {
+                rc = gms::report_cuda_error(e);
+                break;
+            }
+            rc = gms::manifest_launch_window(m, w, p->dev[d], next_launch == 0, d_block_digests, d_tensor_digests, s);
+            if (rc == GMS_OK && (e = cudaEventRecord(p->consumed[d], s)) != cudaSuccess) rc = gms::report_cuda_error(e);
+            ++p->dev_uses;
+        } else {
+            rc = gms::manifest_launch_window(m, windows[next_launch], static_cast<const uint8_t *>(p->dview[b]) + shifts[next_launch],
+                                             next_launch == 0, d_block_digests, d_tensor_digests, s);
+            if (rc == GMS_OK) {
+                cudaError_t e = cudaEventRecord(p->done[b], s);
+                if (e != cudaSuccess) rc = gms::report_cuda_error(e);
+            }
         }
         ++next_launch;
     }
@@ -352,8 +461,13 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
         std::unique_lock<std::mutex> l(reads[w].mu);
         reads[w].cv.wait(l, [&] { return reads[w].pending == 0; });
     }
-    cudaError_t e = cudaStreamSynchronize(s);
+    if (dfd >= 0) close(dfd);
+    cudaError_t e = staged ? cudaStreamSynchronize(p->copy_stream) : cudaSuccess;
     if (e != cudaSuccess && rc == GMS_OK) rc = gms::report_cuda_error(e);
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess && rc == GMS_OK) rc = gms::report_cuda_error(e);
+    st.direct_io = dfd >= 0 && direct_ok.load() ? 1u : 0u;
+    st.copy_engine = staged ? 1u : 0u;
     st.total_seconds = now_s() - t_start;
     if (stats) *stats = st;
     if (io_error) return GMS_ERR_IO;

@@ -176,7 +176,8 @@ def test_kv_pool_shaped_image_is_a_subset_copy_between_pools(oracle):
 @pytest.mark.gpu
 def test_capture_full_size_8b_round_trip(oracle):
     """At the benchmark's size: capture the 16 GB of allocations into an image, then check every image byte with
-    torch, sampled block digests with the oracle, and that the digests equal those of digest-in-place."""
+    torch, every block and tensor digest with the oracle (dealt out to one thread per host core), that digest in
+    place reports the same, and that restoring the captured image gives back the allocations and the digests."""
     w = W.llama3_8b_manifest()
     slab = torch.empty(w.slab_bytes, dtype=torch.uint8, device="cuda")
     W.fill_random_device(slab, 4321)
@@ -189,15 +190,21 @@ def test_capture_full_size_8b_round_trip(oracle):
     for r in w.rows:
         s, o, n = int(r["src_offset"]), int(r["dst_offset"]), int(r["nbytes"])
         assert torch.equal(image[s:s + n], slab[o:o + n])
-    bd2, td2 = d.digest()
-    assert np.array_equal(bd, bd2) and np.array_equal(td, td2)
+    from oracle_threads import all_digests
+
     rec = oracle_record(oracle, w)
-    base, _ = oracle.block_bases(rec)
-    rng = np.random.default_rng(3)
-    for _ in range(300):
-        t = int(rng.integers(0, len(w.rows)))
-        n, o = int(w.rows[t]["nbytes"]), int(w.rows[t]["dst_offset"])
-        b = int(rng.integers(0, (n + 4095) // 4096))
-        want = oracle.block_digest(slab[o + b * 4096:o + min(n, b * 4096 + 4096)].cpu().numpy())
-        assert int(bd[int(base[t]) + b]) == want
+    slab_h = slab.cpu().numpy()
+    obd, otd = all_digests(oracle, rec, lambda t: slab_h[int(w.rows[t]["dst_offset"]):][:int(w.rows[t]["nbytes"])])
+    del slab_h
+    assert np.array_equal(bd, obd) and np.array_equal(td, otd)
+    bd2, td2 = d.digest()
+    assert np.array_equal(bd2, obd) and np.array_equal(td2, otd)
+    # round trip: wipe the allocations, restore them from the captured image
+    want = slab.clone()
+    for r in w.rows:  # the allocations only: the bytes between them belong to nobody and restore leaves them alone
+        o, n = int(r["dst_offset"]), int(r["nbytes"])
+        slab[o:o + n] = 0
+    bd3, td3 = d.restore()
+    assert torch.equal(slab, want)
+    assert np.array_equal(bd3, obd) and np.array_equal(td3, otd)
     d.close()

@@ -1,13 +1,14 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times (library
-defaults).  The oracle cannot redo 16-60 GB in seconds, so each test combines
+defaults).  Every digest the library reports is compared with the oracle's: the single-threaded
+oracle does about 1.1 GB/s per core, so its calls are dealt out to one thread per host core
+(tests/oracle_threads.py) and the 16-34 GB workloads take it a few seconds.  Each test combines
   * exact whole-output properties checked on the device with plain torch ops (every destination
-    byte equals its image byte, nothing else in the slab/pool changed, digest-in-place equals the
-    fused digest), with
-  * oracle values for sampled outputs: whole tensors where they are small enough (or ~1 GB once),
-    and individual 4 KiB blocks drawn from the large ones,
+    byte equals its image byte, nothing else in the slab/pool changed), with
+  * the oracle's block and tensor (or KV-block) digests of the whole workload, compared as entire
+    arrays,
   * host-made single-bit flips that gms_verify must name exactly.
-The mixed manifest (2.3 GB) is checked against the oracle in full, in both its 16-byte-rounded and
-raw odd-sized forms."""
+The mixed manifest (2.3 GB) also goes through the oracle's restore itself, in both its
+16-byte-rounded and raw odd-sized forms."""
 import numpy as np
 import pytest
 
@@ -19,6 +20,7 @@ from paper_2609_25451_b200 import gms  # noqa: E402
 from paper_2609_25451_b200 import workloads as W  # noqa: E402
 
 from gpu_harness import FILL, DeviceWorkload, oracle_record  # noqa: E402
+from oracle_threads import all_digests, all_kv_digests  # noqa: E402
 
 
 def u64(t):
@@ -57,24 +59,22 @@ def test_llama3_8b_manifest_full_size(oracle):
     exp = expected_slab(w, image)
     assert torch.equal(d.slab, exp)
     del exp
-    # digest in place == fused digest (all 3.9 M blocks, all 291 tensors)
-    bd2, td2 = d.digest()
-    assert np.array_equal(bd, bd2) and np.array_equal(td, td2)
-    # oracle: every small tensor whole, one ~1 GB tensor whole, sampled blocks elsewhere
+    # the oracle's digests of the whole image: all 3,921,026 blocks and all 291 tensors
     rec = oracle_record(oracle, w)
     base, total = oracle.block_bases(rec)
     assert total == bd.size == 3_921_026
-    rng = np.random.default_rng(17)
-    whole = [t for t in range(len(w.rows)) if int(w.rows[t]["nbytes"]) <= (16 << 20)][:80] + [0]
-    for t in whole:
-        s, n = int(w.rows[t]["src_offset"]), int(w.rows[t]["nbytes"])
-        T, obd = oracle.tensor_digest(image[s:s + n].cpu().numpy())
-        assert int(td[t]) == T, t
-        assert np.array_equal(bd[int(base[t]):int(base[t]) + obd.size], obd), t
-    check_sampled_blocks(oracle, w, image, bd, base, rng, 400)
+    image_h = image.cpu().numpy()
+    obd, otd = all_digests(oracle, rec, lambda t: image_h[int(w.rows[t]["src_offset"]):][:int(w.rows[t]["nbytes"])])
+    del image_h
+    assert np.array_equal(bd, obd) and np.array_equal(td, otd)
+    # digest in place reports the same, and so do the fused calls
+    bd2, td2 = d.digest()
+    assert np.array_equal(bd2, obd) and np.array_equal(td2, otd)
     # verify: clean, then 3 host-made single-bit flips
     gms.gms_manifest_set_expected(d.m, d.bd_ptr())
     assert d.verify(cap=8) == (0, [])
+    fbd, ftd, fcount, fpairs = d.fused(8)
+    assert np.array_equal(fbd, obd) and np.array_equal(ftd, otd) and (fcount, fpairs) == (0, [])
     flips = W.flip_positions(w, 3, seed=23)
     for row, byte, bit in flips:
         d.flip(row, byte, bit)
@@ -82,9 +82,20 @@ def test_llama3_8b_manifest_full_size(oracle):
     count, pairs = d.verify(cap=8)
     want = sorted(((row, byte // 4096) for row, byte, _ in flips))
     assert count == 3 and pairs == [(int(w.rows[r]["tensor_id"]), b) for r, b in want]
+    ocount, omm = oracle.verify(rec, bd3, obd, 8)  # the oracle's verdict on the same two digest arrays
+    assert ocount == 3 and pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm]
     changed = np.nonzero(bd3 != bd)[0].tolist()
     assert changed == [int(base[r]) + b for r, b in want]
     assert sorted(np.nonzero(td3 != td)[0].tolist()) == sorted({r for r, _ in want})
+    # the damaged blocks' digests are the oracle's digests of the damaged bytes
+    for r, b in want:
+        n, o = int(w.rows[r]["nbytes"]), int(w.rows[r]["dst_offset"])
+        assert int(bd3[int(base[r]) + b]) == oracle.block_digest(d.slab[o + b * 4096:o + min(n, b * 4096 + 4096)].cpu().numpy())
+    fbd, ftd, fcount, fpairs = d.fused(8)
+    assert np.array_equal(fbd, bd3) and np.array_equal(ftd, td3) and (fcount, fpairs) == (3, pairs)
+    # restore + verify in one pass repairs the damage and reports the oracle's digests again
+    fbd, ftd, fcount, fpairs = d.fused(8, restore=True)
+    assert np.array_equal(fbd, obd) and np.array_equal(ftd, otd) and (fcount, fpairs) == (0, [])
     d.close()
 
 
@@ -227,20 +238,37 @@ def test_kv_pool_full_size(oracle):
     untouched = torch.ones(k.n_planes, k.n_blocks, dtype=torch.bool, device="cuda")
     untouched[:, ids.long()] = False
     assert torch.equal(sums_after.view(k.n_planes, k.n_blocks)[untouched], sums_before.view(k.n_planes, k.n_blocks)[untouched])
-    # oracle on sampled slots: all 64 planes of the slot, its 512 block digests and its KV-block digest
-    bd_h, kd_h = u64(bd).reshape(n_sel, k.n_planes, kk), u64(kd)
-    rng = np.random.default_rng(29)
-    for j in rng.choice(n_sel, size=40, replace=False).tolist() + [0, n_sel - 1]:
-        planes = img3[:, j, :].cpu().numpy()
-        T, obd = oracle.tensor_digest(planes.reshape(-1))
-        assert int(kd_h[j]) == T and np.array_equal(bd_h[j].reshape(-1), obd), j
+    # the oracle on every slot: all 1,464,832 block digests and all 2,861 KV-block digests
+    img_h = image.cpu().numpy().reshape(k.n_planes, n_sel, k.block_bytes)
+    obd, okd = all_kv_digests(oracle, n_sel, k.n_planes, k.block_bytes, lambda j: np.ascontiguousarray(img_h[:, j, :]).reshape(-1))
+    del img_h
+    assert obd.size == 1_464_832
+    assert np.array_equal(u64(bd), obd) and np.array_equal(u64(kd), okd)
     # digesting the same blocks where they now lie gives the same digests and writes nothing
     bd2, kd2 = torch.zeros_like(bd), torch.zeros_like(kd)
     gms.gms_kv_digest(desc, ids, n_sel, bd2, kd2, st)
     torch.cuda.synchronize()
     assert st[:2].tolist() == [0, 0]
-    assert torch.equal(bd2, bd) and torch.equal(kd2, kd)
+    assert np.array_equal(u64(bd2), obd) and np.array_equal(u64(kd2), okd)
     assert torch.equal(pool.view(torch.int64).view(k.n_planes * k.n_blocks, -1).sum(dim=1), sums_after)
+    # nothing to report; then one host-made flip, named by block id, plane and sub-block as the oracle names it
+    out = torch.zeros(2 * 8, dtype=torch.int64, device="cuda")
+    cnt = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    scratch = torch.zeros(gms.kv_verify_scratch_words(obd.size), dtype=torch.int32, device="cuda")
+    gms.gms_kv_verify(desc, ids, n_sel, bd2, bd, out, 8, cnt, scratch)
+    torch.cuda.synchronize()
+    assert int(cnt.item()) == 0
+    j, p, c = 1234, 41, 5
+    pos = p * k.plane_stride + int(k.ids[j]) * k.block_stride + c * 4096 + 77
+    pool[pos] = int(pool[pos].item()) ^ 0x02
+    gms.gms_kv_digest(desc, ids, n_sel, bd2, kd2, st)
+    gms.gms_kv_verify(desc, ids, n_sel, bd2, bd, out, 8, cnt, scratch)
+    torch.cuda.synchronize()
+    ocount, orecs = oracle.kv_verify(k.n_planes, k.n_blocks, k.block_bytes, k.ids, u64(bd2), obd, 8)
+    assert int(cnt.item()) == ocount == 1
+    got = out[:2].cpu().numpy().view(gms.KV_MISMATCH_DTYPE)[0]
+    assert tuple(int(got[f]) for f in ("block_id", "plane", "sub_block", "list_pos")) == (int(k.ids[j]), p, c, j)
+    assert tuple(int(orecs[0][f]) for f in ("block_id", "plane", "sub_block", "list_pos")) == (int(k.ids[j]), p, c, j)
 
 
 def test_host_sourced_70b_shard_full_size(oracle):
@@ -268,23 +296,25 @@ def test_host_sourced_70b_shard_full_size(oracle):
             covered[dd:dd + n] = True
         assert bool((slab[~covered] == FILL).all())
         del covered
-        bd2, td2 = d.digest()
-        assert np.array_equal(bd, bd2) and np.array_equal(td, td2)
+        # the oracle's digests of the whole 34.3 GB host image: every block and every one of the 1,413 tensors
         rec = oracle_record(oracle, w)
-        base, _ = oracle.block_bases(rec)
-        rng = np.random.default_rng(31)
-        small = [t for t in range(len(w.rows)) if int(w.rows[t]["nbytes"]) <= (4 << 20)]
-        for t in rng.choice(small, size=60, replace=False).tolist():
-            s, n = int(w.rows[t]["src_offset"]), int(w.rows[t]["nbytes"])
-            T, obd = oracle.tensor_digest(arr[s:s + n])
-            assert int(td[t]) == T and np.array_equal(bd[int(base[t]):int(base[t]) + obd.size], obd), t
-        live = np.nonzero(w.rows["nbytes"] > 0)[0]
-        for _ in range(300):
-            t = int(rng.choice(live))
-            n, s = int(w.rows[t]["nbytes"]), int(w.rows[t]["src_offset"])
-            b = int(rng.integers(0, (n + 4095) // 4096))
-            want = oracle.block_digest(arr[s + b * 4096:s + min(n, b * 4096 + 4096)])
-            assert int(bd[int(base[t]) + b]) == want, (t, b)
+        obd, otd = all_digests(oracle, rec, lambda t: arr[int(w.rows[t]["src_offset"]):][:int(w.rows[t]["nbytes"])])
+        assert np.array_equal(bd, obd) and np.array_equal(td, otd)
+        bd2, td2 = d.digest()
+        assert np.array_equal(bd2, obd) and np.array_equal(td2, otd)
+        # the copy-engine-fed restore of the same image reports the same
+        stage = gms.gms_stage_create(3, 64 << 20)
+        slab.fill_(FILL)
+        d.reset_outputs()
+        gms.gms_restore_staged(d.m, stage, hptr, d.bd_ptr(), d.td_ptr())
+        torch.cuda.synchronize()
+        from gpu_harness import payload_of
+
+        assert np.array_equal(payload_of(d.bd, d.nb), obd) and np.array_equal(payload_of(d.td, d.nt), otd)
+        assert gms.gms_last_device_status(d.m) == 0
+        bd3, td3 = d.digest()  # the bytes it left are the bytes the oracle digested
+        assert np.array_equal(bd3, obd) and np.array_equal(td3, otd)
+        stage.close()
         d.close()
     finally:
         torch.cuda.synchronize()

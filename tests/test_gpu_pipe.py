@@ -1,8 +1,9 @@
-"""gms_restore_fd: restore fed from a file through a ring of pinned buffers.  The result must be
-exactly what gms_restore produces from the same bytes, so the oracle's restore of the file's
-contents is the reference: destination bytes, block digests, tensor digests, bit-exact -- with
-buffers far smaller than the tensors (tensors span many windows), a non-zero file offset, odd
-sizes, and the error paths (short file, bad arguments)."""
+"""gms_restore_fd: restore fed from a file through a ring of pinned buffers and the copy engine.  The
+result must be exactly what gms_restore produces from the same bytes, so the oracle's restore of the
+file's contents is the reference: destination bytes, block digests, tensor digests, bit-exact -- with
+buffers far smaller than the tensors (tensors span many windows), file offsets that are 4 KiB-aligned
+(windows read with O_DIRECT where the file system takes it), 16-byte-aligned and odd, odd sizes, and
+the error paths (short file, bad arguments)."""
 import ctypes
 import os
 
@@ -26,6 +27,7 @@ def test_pipe_argument_checks_need_no_gpu():
     assert L.gms_pipe_create(2, 1 << 20, 0, ctypes.byref(out)) == gms.ERR_ARG       # no readers
     assert L.gms_pipe_create(2, 1 << 20, 4, None) == gms.ERR_NULL
     assert L.gms_pipe_destroy(None) == gms.OK
+    assert L.gms_pipe_direct_io(None, 1) == gms.ERR_NULL
     assert L.gms_restore_fd(None, None, 0, 0, None, None, None, None) == gms.ERR_NULL
     assert "file" in gms.gms_strerror(gms.ERR_IO)
 
@@ -37,7 +39,8 @@ def _write_image(path, image: np.ndarray, file_offset: int):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("n_buffers,buffer_mib,n_readers,file_offset", [(2, 1, 1, 0), (3, 2, 4, 4096 + 16), (4, 16, 8, 512)])
+@pytest.mark.parametrize("n_buffers,buffer_mib,n_readers,file_offset",
+                         [(2, 1, 1, 0), (3, 2, 4, 4096 + 16), (4, 16, 8, 512), (3, 4, 6, 8192), (2, 2, 3, 5)])
 def test_restore_fd_equals_restore_of_the_same_bytes(oracle, tmp_path, n_buffers, buffer_mib, n_readers, file_offset):
     w = W.mixed_manifest(n_small=1500, n_large=3, large_bytes=(7 << 20) + 40, round16=False, seed=123)
     image = W.random_bytes_host(w.image_bytes, seed=77)
@@ -50,7 +53,8 @@ def test_restore_fd_equals_restore_of_the_same_bytes(oracle, tmp_path, n_buffers
     pipe = gms.gms_pipe_create(n_buffers, buffer_mib << 20, n_readers)
     fd = os.open(path, os.O_RDONLY)
     try:
-        for _ in range(2):  # twice: the second call must not be disturbed by what the first left in the buffers
+        for direct in (False, True):  # twice: the second call must not be disturbed by what the first left in the buffers
+            gms.gms_pipe_direct_io(pipe, direct)  # second pass: O_DIRECT reads where the file system takes them
             d.slab.fill_(FILL)
             d.reset_outputs()
             st = gms.gms_restore_fd(d.m, pipe, fd, file_offset, d.bd_ptr(), d.td_ptr())
@@ -60,6 +64,8 @@ def test_restore_fd_equals_restore_of_the_same_bytes(oracle, tmp_path, n_buffers
             assert np.array_equal(d.slab_host(), slab_h), "destination bytes (or guard bands) differ"
             assert np.array_equal(payload_of(d.bd, d.nb), obd) and np.array_equal(payload_of(d.td, d.nt), otd)
             assert st["windows"] >= w.image_bytes // (buffer_mib << 20) and st["bytes_read"] <= w.image_bytes
+            # windows go through the copy engine; whether reads bypass the page cache is up to the file system
+            assert st["copy_engine"] == 1 and st["direct_io"] in ((0, 1) if direct else (0,))
     finally:
         os.close(fd)
         pipe.close()
