@@ -4,7 +4,8 @@
 
 Draws random manifests (counts, size mixes, alignments, chunk lengths), random operations
 (restore from device / mapped host / staged host image, digest, capture, verify after random
-host-made corruption, KV restore / capture with random ids) and compares every output with the
+host-made corruption -- as separate calls and as the fused gms_digest_verify / gms_restore_verify --,
+KV restore / capture / digest / verify with random ids) and compares every output with the
 CPU oracle, bit for bit.  Prints one line per 50 iterations and exits non-zero on the first
 difference."""
 import argparse
@@ -85,7 +86,22 @@ def one_manifest_round(rng, it):
     cap = int(rng.choice([0, 1, 3, 64]))
     count, pairs = d.verify(cap=cap)
     ocount, omm = oracle.verify(rec, obd2, obd, cap=cap)
-    assert count == ocount and pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm], "verify differs"
+    want_pairs = [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+    assert count == ocount and pairs == want_pairs, "verify differs"
+    # the same through the fused calls: digest + verify in one pass, then restore + verify against damaged records
+    fbd, ftd, fcount, fpairs = d.fused(cap)
+    assert np.array_equal(fbd, obd2) and np.array_equal(ftd, otd2) and (fcount, fpairs) == (ocount, want_pairs), "digest_verify differs"
+    if rng.integers(0, 2):
+        gms.gms_manifest_set_expected(d.m, d.bd_ptr())  # records of the damaged state
+        fbd, ftd, fcount, fpairs = d.fused(cap, restore=True)
+        ocount3, omm3 = oracle.verify(rec, obd, obd2, cap=cap)
+        assert np.array_equal(fbd, obd) and np.array_equal(ftd, otd), "restore_verify digests differ"
+        assert (fcount, fpairs) == (ocount3, [(int(m["tensor_id"]), int(m["block"])) for m in omm3]), "restore_verify list differs"
+        slab_h2 = np.full(w.slab_bytes, FILL, np.uint8)
+        oracle.restore(rec, image, slab_h2)
+        assert np.array_equal(d.slab_host(), slab_h2), "restore_verify bytes differ"
+        slab_h = slab_h2
+        obd2, otd2 = obd, otd
     # capture the (corrupted) allocations back and compare with the oracle's capture
     want_img = np.full(w.image_bytes, 0x3C, np.uint8)
     oracle.capture(rec, want_img, slab_h)
@@ -145,6 +161,33 @@ def one_kv_round(rng):
     assert int(status[0]) == oskip2 and int(status[1]) == 0, "kv digest status differs"
     assert np.array_equal(pool.cpu().numpy(), want_pool), "kv digest wrote to the pool"
     assert np.array_equal(payload_of(bd, n_sel * n_planes * k), obd2) and np.array_equal(payload_of(kd, n_sel), okd2), "kv in-place digests"
+    # host-made damage in the pool, digest again, and gms_kv_verify against the oracle's kv_verify
+    n_slots = n_sel * n_planes * k
+    expected = payload_of(bd, n_slots)
+    exp_d = torch.from_numpy(expected.view(np.int64).copy()).cuda()
+    pool_h2 = pool.cpu().numpy()
+    for _ in range(int(rng.integers(0, 5))):
+        pool_h2[int(rng.integers(0, pool_h2.size))] ^= 1 << int(rng.integers(0, 8))
+    pool.copy_(torch.from_numpy(pool_h2))
+    gms.gms_kv_digest(desc, ids_d, n_sel, bd.data_ptr() + 8 * PAD, kd.data_ptr() + 8 * PAD, st.data_ptr() + 8 * PAD)
+    torch.cuda.synchronize()
+    computed = payload_of(bd, n_slots)
+    rc, obd3, _, _ = oracle.kv_digest(pool_h2, plane_stride, bb, n_planes, n_blocks, bb, ids)
+    assert rc == 0 and np.array_equal(computed, obd3), "kv digests of the damaged pool"
+    cap = int(rng.choice([0, 1, 4, 64]))
+    out = torch.full((2 * cap + 2 * PAD,), CANARY, dtype=torch.int64, device="cuda")
+    cnt = guarded_u64(1)
+    scratch = torch.zeros(gms.kv_verify_scratch_words(n_slots), dtype=torch.int32, device="cuda")
+    gms.gms_kv_verify(desc, ids_d, n_sel, bd.data_ptr() + 8 * PAD, exp_d, out.data_ptr() + 8 * PAD, cap, cnt.data_ptr() + 8 * PAD, scratch)
+    torch.cuda.synchronize()
+    ocount, orecs = oracle.kv_verify(n_planes, n_blocks, bb, ids, computed, expected, cap)
+    count = int(payload_of(cnt, 1)[0])
+    words = payload_of(out, 2 * cap)
+    kk = min(count, cap)
+    assert count == ocount and (words[2 * kk:] == CANARY).all(), "kv verify count"
+    got = words[: 2 * kk].view(gms.KV_MISMATCH_DTYPE)
+    f = ("block_id", "plane", "sub_block", "list_pos")
+    assert [tuple(int(r[x]) for x in f) for r in got] == [tuple(int(r[x]) for x in f) for r in orecs], "kv verify records"
 
 
 def main():
