@@ -510,8 +510,6 @@ int gms_service_back_pages(gms_service *s);
  *       (defaults 1,1 / 2,1; counters 1..32, chunks 1..64)
  *   GMS_CHUNK_BLOCKS / GMS_CHUNK_BLOCKS_DIGEST         4 KiB blocks per chunk of the copy list and of the digest
  *       list (defaults 4 / 8, fewer for small manifests; 1..32)
- *   GMS_L2_HINTS                                       L2 eviction hints of the bulk copies, bits 0-1 loads and
- *       2-3 stores: 0 none (default), 1 evict_first, 2 evict_last
  */
 
 /* Launch geometry of the streaming kernels on the current device (for reporting). */

@@ -173,7 +173,6 @@ int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void
     a.n_tensors = (uint32_t)m->entries.size();
     a.work_counters = m->d_counter;
     a.status = m->d_status;
-    a.hints = 0;
     a.n_counters = 1;
     a.group = 1;
     a.capture = 0;
@@ -400,7 +399,6 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
     a.n_tensors = (uint32_t)m->entries.size();
     a.work_counters = m->d_counter;
     a.status = m->d_status;
-    a.hints = 0;
     a.n_counters = 1;
     a.group = 1;
     a.capture = capture ? 1u : 0u;
@@ -586,7 +584,6 @@ static int kv_call(const gms_kv_pool *pool, const void *image, uint64_t img_plan
     a.block_digests = d_block_digests;
     a.kv_digests = d_kv_digests;
     a.status = reinterpret_cast<unsigned long long *>(d_status);
-    a.hints = 0;
     a.capture = capture ? 1u : 0u;
     a.digest_only = 0u;
     a.by_id = (pool->flags & GMS_KV_IMAGE_BY_ID) ? 1u : 0u;

@@ -35,7 +35,6 @@ struct Geometry {
     uint32_t warps;    // warps per CTA; every warp runs its own copy pipeline
     uint32_t stages;   // 4 KiB ring slots per warp
     uint32_t smem;     // dynamic shared memory per CTA
-    uint32_t hints;    // L2 eviction hints of the bulk copies: bits 0-1 loads, bits 2-3 stores (0 = none)
     uint32_t counters; // work counters the chunk claims are spread over
     uint32_t group;    // consecutive chunks bought by one claim
 };
@@ -51,7 +50,6 @@ struct StreamArgs {
     uint32_t n_tensors;
     unsigned int *work_counters;   // manifest-owned: kMaxCounters counters, kCounterStride words apart
     unsigned long long *status;    // manifest-owned device status word
-    uint32_t hints;                // filled in by the launcher
     uint32_t n_counters;           // filled in by the launcher
     uint32_t group;                // filled in by the launcher
     uint32_t capture;              // 1: gather allocations into the image (restore kernel with roles swapped)
@@ -76,7 +74,6 @@ struct KvArgs {
     uint32_t capture;              // 1: gather pool blocks into the image
     uint32_t digest_only;          // 1: digest the selected pool blocks where they lie (no image, nothing written)
     uint32_t by_id;               // 1: the image is pool-shaped (slot = block id), else packed (slot = list position)
-    uint32_t hints;                // filled in by the launcher
 };
 
 cudaError_t launch_restore(const StreamArgs &a, cudaStream_t s);

@@ -134,12 +134,6 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------- digest arithmetic
-__device__ __forceinline__ uint64_t mix_full(uint64_t z)
-{
-    z = (z ^ (z >> 30)) * kM1;
-    z = (z ^ (z >> 27)) * kM2;
-    return z ^ (z >> 31);
-}
 // Three-input XOR in one LOP3.
 __device__ __forceinline__ uint32_t xor3(uint32_t a, uint32_t b, uint32_t c)
 {
@@ -170,38 +164,19 @@ __device__ __forceinline__ void mix_head32(uint32_t lo, uint32_t hi, uint32_t cl
     const uint32_t ul = zl ^ __funnelshift_r(zl, zh, 27), uh = zh ^ (zh >> 27);
     mul64_lo(ul, uh, M2l, M2h, ql, qh);
 }
+// The whole mix, for the tensor digest (once per block digest).
+__device__ __forceinline__ uint64_t mix_full32(uint64_t z)
+{
+    uint32_t ql, qh;
+    mix_head32((uint32_t)z, (uint32_t)(z >> 32), 0u, 0u, ql, qh);
+    const uint64_t y = ((uint64_t)qh << 32) | ql;
+    return y ^ (y >> 31);
+}
 __device__ __forceinline__ uint64_t warp_xor64(uint64_t v)
 {
     uint32_t lo = __reduce_xor_sync(kFull, (uint32_t)v);
     uint32_t hi = __reduce_xor_sync(kFull, (uint32_t)(v >> 32));
     return ((uint64_t)hi << 32) | lo;
-}
-
-// Bulk copies with an L2 eviction-priority hint (the payload is touched exactly once).
-__device__ __forceinline__ uint64_t l2_policy(uint32_t code)  // 1 evict_first, 2 evict_last, else evict_normal
-{
-    uint64_t pol;
-    if (code == 1)
-        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    else if (code == 2)
-        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    else
-        asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar, uint64_t pol)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
-                     dst_smem),
-                 "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar), "l"(pol)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_store_hint(void *dst, uint32_t src_smem, uint32_t bytes, uint64_t pol)
-{
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(
-                     __cvta_generic_to_global(dst)),
-                 "r"(src_smem), "r"(bytes), "l"(pol)
-                 : "memory");
 }
 
 // ---------------------------------------------------------------- chunk providers (warp-uniform)
@@ -361,8 +336,8 @@ struct KvProvider {
 // while the digest is still in a register, so that gms_digest_verify / gms_restore_verify only run scan + emit.
 template <int S, bool kStore, class Provider>
 __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint4 *fifo, uint64_t *bars, uint64_t *block_digests,
-                                             uint64_t *accum, unsigned long long *status, uint32_t hints,
-                                             const uint64_t *expected, uint32_t *seg_count)
+                                             uint64_t *accum, unsigned long long *status, const uint64_t *expected,
+                                             uint32_t *seg_count)
 {
     static_assert(S <= (int)kFifo, "the chunk fifo must cover the ring");
     constexpr uint32_t LOOK = S - 1;  // blocks in flight ahead of the one being digested
@@ -381,8 +356,6 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
         }
 
     const uint32_t ring_s = smem_u32(ring), bars_s = smem_u32(bars);
-    const uint32_t ld_hint = hints & 3u, st_hint = (hints >> 2) & 3u;
-    const uint64_t ld_pol = l2_policy(ld_hint), st_pol = l2_policy(st_hint);
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < S; ++s) mbar_init(bars_s + 8u * s, 1u);
@@ -398,14 +371,14 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
     // issue-side cursor (the chunk being fetched) and digest-side cursor (the chunk being consumed);
     // chunk records travel from one to the other through a small per-warp fifo in shared memory
     Item it{};
-    uint32_t it_blocks = 0, it_next = 0, chunks_in = 0;
+    uint32_t it_blocks = 0, it_full = 0, it_next = 0, chunks_in = 0, stall_extra = 0;
     uint64_t c_dst = 0;
     uint32_t c_nbytes = 0, c_tensor = 0, c_gblock0 = 0, c_tblock0 = 0, c_blocks = 0, c_next = 0, chunks_out = 0;
     bool more = true, failed = false;
     uint32_t issued = 0, consumed = 0;
     uint32_t is = 0;               // ring slot of the next block to issue   (issued % S)
     uint32_t cs = 0, cparity = 0;  // ring slot and barrier phase of the next block to digest
-    uint64_t myD = 0;
+    uint32_t my_lo = 0, my_hi = 0;
     // share of a tensor digest gathered over consecutive chunks of the same tensor: one atomic per run, not per chunk
     uint32_t run_tensor = 0xffffffffu;
     uint64_t run_val = 0;
@@ -417,6 +390,8 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
                 more = prov.next(it, lane);
                 if (!more) break;
                 it_blocks = (it.nbytes + kBlockBytes - 1) >> 12;
+                it_full = it.nbytes >> 12;  // whole blocks: nothing to pad, no hand-moved tail
+                stall_extra = it.stall;     // self-test only: announced on the chunk's first barrier, never sent
                 it_next = 0;
                 if (lane == 0) {
                     const uint64_t d = reinterpret_cast<uint64_t>(it.dst);
@@ -428,13 +403,14 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
             const uint32_t s = is;
             is = (is + 1 == S) ? 0 : is + 1;
             const uint32_t off = it_next << 12;
-            const uint32_t m = min(kBlockBytes, it.nbytes - off);
-            const uint32_t m16 = m & ~15u;
-            uint8_t *stage = ring + s * kBlockBytes;
             // the slot was last read by the store of block issued-S: all but the newest group must have read
             if (kStore && lane == 0) bulk_wait_read<S - LOOK>();
-            if (m < kBlockBytes) {
+            uint32_t m16 = kBlockBytes;
+            if (it_next >= it_full) {
                 // short last block of a tensor: zero-fill the slot past the bulk part and move the <16 B tail by hand
+                const uint32_t m = it.nbytes - off;
+                m16 = m & ~15u;
+                uint8_t *stage = ring + s * kBlockBytes;
                 __syncwarp();
                 for (uint32_t o = m16 + 16u * lane; o < kBlockBytes; o += 512u)
                     *reinterpret_cast<uint4 *>(stage + o) = make_uint4(0, 0, 0, 0);
@@ -448,14 +424,10 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
                 __syncwarp();
             }
             if (lane == 0) {
-                mbar_arrive_expect_tx(bars_s + 8u * s, m16 + (it_next == 0 ? it.stall : 0u));
-                if (m16) {
-                    if (ld_hint)
-                        bulk_load_hint(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s, ld_pol);
-                    else
-                        bulk_load(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s);
-                }
+                mbar_arrive_expect_tx(bars_s + 8u * s, m16 + stall_extra);
+                if (m16) bulk_load(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s);
             }
+            stall_extra = 0;
             ++it_next;
             ++issued;
         }
@@ -485,12 +457,7 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
         if (kStore && lane == 0) {
             const uint32_t off = c_next << 12;
             const uint32_t m16 = min(kBlockBytes, c_nbytes - off) & ~15u;
-            if (m16) {
-                if (st_hint)
-                    bulk_store_hint(reinterpret_cast<void *>(c_dst + off), ring_s + s * kBlockBytes, m16, st_pol);
-                else
-                    bulk_store(reinterpret_cast<void *>(c_dst + off), ring_s + s * kBlockBytes, m16);
-            }
+            if (m16) bulk_store(reinterpret_cast<void *>(c_dst + off), ring_s + s * kBlockBytes, m16);
             bulk_commit();
         }
         uint32_t al = 0, ah = 0;
@@ -503,15 +470,17 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
             al = xor3(al, pl, ql);
             ah = xor3(ah, ph, qh);
         }
-        const uint64_t acc = ((uint64_t)__reduce_xor_sync(kFull, ah) << 32) | __reduce_xor_sync(kFull, al);
-        if (lane == c_next) myD = acc ^ (acc >> 31);
+        al = __reduce_xor_sync(kFull, al);
+        ah = __reduce_xor_sync(kFull, ah);
+        if (lane == c_next) my_lo = al, my_hi = ah;  // the block's XOR before the last xor-shift, which waits for the chunk's end
         ++c_next;
         if (c_next == c_blocks) {  // chunk complete: block digests leave coalesced, one atomic for the tensor digest
             uint64_t t = 0;
             if (lane < c_blocks) {
+                const uint64_t raw = ((uint64_t)my_hi << 32) | my_lo, myD = raw ^ (raw >> 31);
                 if (block_digests) block_digests[(uint64_t)c_gblock0 + lane] = myD;
                 if (expected && __ldg(expected + c_gblock0 + lane) != myD) atomicAdd(seg_count + ((c_gblock0 + lane) >> kVerifySegShift), 1u);
-                t = mix_full(myD ^ ((uint64_t)(c_tblock0 + lane) * kG));
+                t = mix_full32(myD ^ ((uint64_t)(c_tblock0 + lane) * kG));
             }
             t = warp_xor64(t);
             if (c_tensor != run_tensor) {
@@ -575,7 +544,7 @@ __global__ void __launch_bounds__(512, 1) gms_stream_kernel(StreamArgs a)
     // whatever follows on the stream may be scheduled now; every kernel of this library waits (griddepcontrol.wait)
     // for the grid before it to finish before it touches global memory
     asm volatile("griddepcontrol.launch_dependents;");
-    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.hints, a.expected,
+    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.expected,
                             a.seg_count);
 }
 
@@ -589,7 +558,7 @@ __global__ void __launch_bounds__(512, 1) gms_kv_stream_kernel(KvArgs a)
     prov.counter = reinterpret_cast<unsigned int *>(a.status + 2);
     prov.total = a.n_sel * a.n_planes;
     asm volatile("griddepcontrol.launch_dependents;");
-    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, a.hints, nullptr, nullptr);
+    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, nullptr, nullptr);
 }
 
 // Clears the accumulators the streaming kernels XOR / add into (and, for the fused compare, the per-segment
@@ -697,7 +666,6 @@ cudaError_t launch_stream(const StreamArgs &a, cudaStream_t s)
         return e;
     if (a.n_chunks == 0) return cudaSuccess;
     StreamArgs b = a;
-    b.hints = g.hints;
     b.n_counters = g.counters;
     // a claim buys a run of chunks only while there are runs enough for every warp
     b.group = (uint32_t)std::min<uint64_t>(g.group, std::max<uint64_t>(1, a.n_chunks / (4ull * g.grid * g.warps)));
@@ -745,8 +713,6 @@ cudaError_t get_geometry(Kind kind, Geometry *out)
         while (g.warps > 1 && (need(g.warps) + 1024) * per_sm > (uint32_t)max_smem) --g.warps;
         g.smem = need(g.warps);
         g.grid = (uint32_t)sms * per_sm;
-        g.hints = 0;
-        if (const char *v = hook("GMS_L2_HINTS")) g.hints = (uint32_t)atoi(v) & 15u;  // bits 0-1 load, 2-3 store
         // claims: the restore kernels draw single chunks from one counter (strict list order keeps the bytes in
         // flight a compact front, which HBM rewards); the digest kernel claims twice as often per second, so it
         // spreads its claims over two counters (one ticket buys one 32 KiB chunk of its own, longer-cut list:
@@ -782,8 +748,7 @@ cudaError_t launch_kv_restore(const KvArgs &a, cudaStream_t s)
     if (e) return e;
     if ((e = prologue(a.kv_digests, a.n_sel, nullptr, 0, a.status, 4, nullptr, 0, s))) return e;
     if (a.n_sel == 0 || a.n_planes == 0) return cudaSuccess;
-    KvArgs b = a;
-    b.hints = g.hints;
+    const KvArgs &b = a;
     if (a.digest_only) {
         switch (g.stages) {
         case 3: e = launch_after_prologue(gms_kv_stream_kernel<3, false>, g, s, b); break;
