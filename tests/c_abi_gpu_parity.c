@@ -127,6 +127,29 @@ int main(void)
     for (i = 0; i < w_count; ++i) CHECK(h_out[i].tensor_id == w_out[i].tensor_id && h_out[i].block == w_out[i].block);
     CHECK(h_out[0].tensor_id == oe[7].tensor_id && h_out[0].block == 1 && h_out[1].tensor_id == oe[30].tensor_id);
 
+    /* the same decision in one pass: gms_digest_verify reports the digests and the list of the two calls above */
+    CHECK(cudaMemset(d_bd, 0, 8 * n_blocks) == cudaSuccess && cudaMemset(d_out, 0, sizeof(gms_mismatch) * CAP) == cudaSuccess);
+    CHECK(gms_digest_verify(m, d_bd, d_td, d_out, CAP, d_count, NULL) == GMS_OK);
+    CHECK(cudaDeviceSynchronize() == cudaSuccess);
+    CHECK(cudaMemcpy(h_bd, d_bd, 8 * n_blocks, cudaMemcpyDeviceToHost) == cudaSuccess);
+    CHECK(cudaMemcpy(&h_count, d_count, 8, cudaMemcpyDeviceToHost) == cudaSuccess);
+    CHECK(cudaMemcpy(h_out, d_out, sizeof h_out, cudaMemcpyDeviceToHost) == cudaSuccess);
+    CHECK(memcmp(h_bd, w_bd2, 8 * n_blocks) == 0 && h_count == w_count);
+    for (i = 0; i < w_count; ++i) CHECK(h_out[i].tensor_id == w_out[i].tensor_id && h_out[i].block == w_out[i].block);
+
+    /* gms_restore_verify puts the image back over the damage: the oracle's restore digests again, nothing differs */
+    CHECK(gms_restore_verify(m, d_image, GMS_SRC_DEVICE, d_bd, d_td, d_out, CAP, d_count, NULL) == GMS_OK);
+    CHECK(cudaDeviceSynchronize() == cudaSuccess);
+    CHECK(gms_last_device_status(m, NULL, &status) == GMS_OK && status == 0);
+    CHECK(cudaMemcpy(h_slab, d_slab, slab_bytes, cudaMemcpyDeviceToHost) == cudaSuccess);
+    CHECK(cudaMemcpy(h_bd, d_bd, 8 * n_blocks, cudaMemcpyDeviceToHost) == cudaSuccess);
+    CHECK(cudaMemcpy(h_td, d_td, 8 * N, cudaMemcpyDeviceToHost) == cudaSuccess);
+    CHECK(cudaMemcpy(&h_count, d_count, 8, cudaMemcpyDeviceToHost) == cudaSuccess);
+    CHECK(gmso_restore(oe, N, h_image, image_bytes, h_want, slab_bytes, w_bd2, w_td2) == 0);
+    CHECK(memcmp(h_slab, h_want, slab_bytes) == 0);
+    CHECK(memcmp(h_bd, w_bd2, 8 * n_blocks) == 0 && memcmp(h_td, w_td2, 8 * N) == 0);
+    CHECK(h_count == gmso_verify(oe, N, w_bd2, w_bd, w_out, CAP) && h_count == 0);
+
     CHECK(gms_manifest_destroy(m) == GMS_OK);
     cudaFree(d_image); cudaFree(d_slab); cudaFree(d_bd); cudaFree(d_td); cudaFree(d_out); cudaFree(d_count);
     printf("c abi gpu parity: ok (%d tensors, %llu blocks, %llu launches)\n", (int)N, (unsigned long long)n_blocks,
