@@ -82,6 +82,67 @@ def test_restore_verify_digest_replay_from_a_graph(oracle):
     d.close()
 
 
+def test_fused_calls_replay_from_a_graph(oracle):
+    """gms_restore_verify + gms_digest_verify captured once (5 kernel nodes less than the separate calls need) and
+    replayed over images that differ from the recorded one in a few blocks: digests, list and count from the oracle."""
+    w = W.mixed_manifest(n_small=2500, n_large=4, large_bytes=(12 << 20) + 24, round16=False, seed=91)  # > 16 K blocks
+    rec = oracle_record(oracle, w)
+    image_a = W.random_bytes_host(w.image_bytes, seed=72)
+    image_b = image_a.copy()
+    for row, byte, bit in W.flip_positions(w, 5, seed=10):
+        image_b[int(w.rows[row]["src_offset"]) + byte] ^= 1 << bit
+
+    def want(image):
+        slab = np.full(w.slab_bytes, FILL, np.uint8)
+        rc, bd, td = oracle.restore(rec, image, slab)
+        assert rc == 0
+        return slab, bd, td
+
+    slab_a, bd_a, td_a = want(image_a)
+    slab_b, bd_b, td_b = want(image_b)
+    d = DeviceWorkload(w, image_a)
+    assert d.nb > 16384  # the emit kernel runs over several segments
+    expected = torch.from_numpy(bd_a.view(np.int64).copy()).cuda()
+    gms.gms_manifest_set_expected(d.m, expected.data_ptr())
+    cap = 16
+    out1 = torch.full((2 * cap + 2 * PAD,), CANARY, dtype=torch.int64, device="cuda")
+    out2 = torch.full((2 * cap + 2 * PAD,), CANARY, dtype=torch.int64, device="cuda")
+    cnt1, cnt2 = guarded_u64(1), guarded_u64(1)
+    bd2, td2 = guarded_u64(d.nb), guarded_u64(d.nt)
+
+    def step():
+        gms.gms_restore_verify(d.m, d.image, gms.SRC_DEVICE, d.bd_ptr(), d.td_ptr(), out1.data_ptr() + 8 * PAD, cap,
+                               cnt1.data_ptr() + 8 * PAD)
+        gms.gms_digest_verify(d.m, bd2.data_ptr() + 8 * PAD, td2.data_ptr() + 8 * PAD, out2.data_ptr() + 8 * PAD, cap,
+                              cnt2.data_ptr() + 8 * PAD)
+
+    _warm(step)
+    launches0 = gms.gms_kernel_launches()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    assert gms.gms_kernel_launches() - launches0 == 6  # per call: prologue, streaming kernel, emit
+
+    for image, slab_w, bd_w, td_w in ((image_b, slab_b, bd_b, td_b), (image_a, slab_a, bd_a, td_a), (image_b, slab_b, bd_b, td_b)):
+        d.image.copy_(torch.from_numpy(image))
+        d.slab.fill_(FILL)
+        for t in (d.bd, d.td, bd2, td2, out1, out2, cnt1, cnt2):
+            t.fill_(CANARY)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert gms.gms_last_device_status(d.m) == 0
+        assert np.array_equal(d.slab_host(), slab_w)
+        ocount, omm = oracle.verify(rec, bd_w, bd_a, cap=cap)
+        want_pairs = [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+        for bdt, tdt, out, cnt in ((d.bd, d.td, out1, cnt1), (bd2, td2, out2, cnt2)):
+            assert np.array_equal(payload_of(bdt, d.nb), bd_w) and np.array_equal(payload_of(tdt, d.nt), td_w)
+            assert int(payload_of(cnt, 1)[0]) == ocount
+            pairs = payload_of(out, 2 * cap).reshape(cap, 2)
+            assert [(int(a), int(b)) for a, b in pairs[:ocount]] == want_pairs and (pairs[ocount:] == CANARY).all()
+    assert ocount == 5
+    d.close()
+
+
 def test_kv_restore_replays_from_a_graph_with_new_block_ids(oracle):
     n_planes, n_blocks, block_bytes, n_sel = 4, 96, 16384, 40
     rng = np.random.default_rng(5)

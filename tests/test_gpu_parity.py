@@ -224,6 +224,22 @@ def test_host_mapped_source_parity(oracle):
         bd, td = d.restore(image=dview, kind=gms.SRC_HOST_MAPPED)
         assert np.array_equal(d.slab_host(), want_slab)
         assert np.array_equal(bd, want_bd) and np.array_equal(td, want_td)
+        # the fused restore + verify reads the mapped image just the same
+        gms.gms_manifest_set_expected(d.m, d.bd_ptr())
+        d.slab.fill_(FILL)
+        d.reset_outputs()
+        out = torch.full((2 * 4,), -1, dtype=torch.int64, device="cuda")
+        cnt = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+        gms.gms_restore_verify(d.m, dview, gms.SRC_HOST_MAPPED, d.bd_ptr(), d.td_ptr(), out, 4, cnt)
+        torch.cuda.synchronize()
+        assert int(cnt.item()) == 0 and (out == -1).all() and np.array_equal(d.slab_host(), want_slab)
+        assert np.array_equal(payload_of(d.bd, d.nb), want_bd) and np.array_equal(payload_of(d.td, d.nt), want_td)
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_restore_verify(d.m, dview, gms.SRC_DEVICE, d.bd_ptr(), d.td_ptr(), out, 4, cnt)
+        assert ei.value.status == gms.ERR_KIND
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_restore_verify(d.m, dview, gms.SRC_HOST_MAPPED, None, d.td_ptr(), out, 4, cnt)
+        assert ei.value.status == gms.ERR_NULL
         # the pointer must be what image_kind says
         with pytest.raises(gms.GmsError) as ei:
             gms.gms_restore(d.m, dview, gms.SRC_DEVICE, None, None)
