@@ -230,6 +230,16 @@ class ManifestBench:
         self.bytes_digest = self.payload + 8 * nb + 32 * n_dchunks
         self.bytes_restore = 2 * self.payload + 8 * nb + 32 * self.n_chunks
         self.bytes_verify = 16 * nb
+        self.set_fused(fused)
+        self.launches_per_step = None
+        self.graph = None
+        # a working set that L2 (126 MB) could hold between steps is flushed out before every step
+        self.l2_flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev) if self.payload < (512 << 20) else None
+
+    def set_fused(self, fused: bool):
+        """Two fused calls per step (digest + verify, restore + verify in one pass each) or the four separate ones."""
+        nb = self.m.n_blocks
+        self.fused = fused
         if fused:
             self.phase_names = ["digest_verify", "restore_verify"]
             self.phase_bytes = {"digest_verify": self.bytes_digest + 8 * nb, "restore_verify": self.bytes_restore + 8 * nb}
@@ -240,10 +250,6 @@ class ManifestBench:
                                 "verify2": self.bytes_verify}
             self.dominant = "restore"
         self.traffic = sum(self.phase_bytes.values())
-        self.launches_per_step = None
-        self.graph = None
-        # a working set that L2 (126 MB) could hold between steps is flushed out before every step
-        self.l2_flush = torch.zeros(256 << 20, dtype=torch.uint8, device=dev) if self.payload < (512 << 20) else None
 
     def use_graph(self):
         """Captures one step into a CUDA graph; later steps replay it (no per-phase times then)."""
@@ -1062,6 +1068,16 @@ def run_file(args, torch, gms, W, dev, index, want_cpu=True):
             os.remove(path)
 
 
+def unfused_comparison(torch, gms, bench, steps, warmup, index):
+    """The same manifest step as four separate calls, on the same buffers (what the fused calls save)."""
+    bench.set_fused(False)
+    ue = measure(torch, gms, bench, steps, warmup, index)
+    bench.set_fused(True)
+    return {"step": ue["step"], "steps": steps, "ms_per_step": ue["ms_per_step"], "parity_ok": ue["parity_ok"],
+            "phases_ms_median": {k: v["median_ms"] for k, v in ue["phases"].items()},
+            "phases_ms_mean": {k: v["mean_ms"] for k, v in ue["phases"].items()}}
+
+
 def release(torch):
     gc.collect()
     torch.cuda.synchronize()
@@ -1186,6 +1202,8 @@ def main():
 
     # ---- all five configurations (single GPU, default invocation only)
     if args.workload is None and world == 1:
+        entry["unfused_step"] = unfused_comparison(torch, gms, bench, min(args.steps, 10), args.warmup, local_rank)
+        line["unfused_step"] = entry["unfused_step"]
         entry["cpu_baseline"] = line.get("cpu_baseline")
         entry["e2e"] = line.get("e2e")
         configs = {"8b": entry}
@@ -1198,15 +1216,11 @@ def main():
             b = build(name)
             steps = 50 if name == "tiny" else args.steps
             e = measure(torch, gms, b, steps, args.warmup, local_rank)
-            if name == "tiny":  # launch- and latency-bound: also the same work as four separate calls
-                u = ManifestBench(name, torch, gms, W, dev, fused=False)
-                ue = measure(torch, gms, u, steps, args.warmup, local_rank)
-                e["unfused_step"] = {"step": ue["step"], "ms_per_step": ue["ms_per_step"], "parity_ok": ue["parity_ok"],
-                                     "phases_ms_median": {k: v["median_ms"] for k, v in ue["phases"].items()}}
+            if name != "kv":  # also the same work as four separate calls
+                e["unfused_step"] = unfused_comparison(torch, gms, b, steps, args.warmup, local_rank)
+            if name == "tiny":
                 e["note"] = ("latency-bound: 67 MB of traffic is 10 us at the HBM rate; what is measured is launch, "
                              "ramp-up and tail of a 148-CTA persistent kernel")
-                u.close()
-                del u
             if want_cpu and name == "kv":
                 e["cpu_baseline"] = cpu_baseline_kv(b.k, lambda n: b.image[:n].cpu().numpy())
             elif want_cpu:
