@@ -213,7 +213,10 @@ class ManifestBench:
         else:
             self.slab = torch.zeros(w.slab_bytes, dtype=torch.uint8, device=dev)
             self.entries = self._entries(self.slab.data_ptr())
+        gms.gms_manifest_build(self.entries[:1], w.image_bytes).close()  # first call on a device sets the launch shapes up
+        t0 = time.perf_counter()
         self.m = gms.gms_manifest_build(self.entries, w.image_bytes)
+        self.build_ms = (time.perf_counter() - t0) * 1e3  # host: validation, work lists, upload of the tables
         self.bd = torch.zeros(max(self.m.n_blocks, 1), dtype=torch.int64, device=dev)
         self.td = torch.zeros(max(self.m.n_tensors, 1), dtype=torch.int64, device=dev)
         self.cap = 64
@@ -495,6 +498,7 @@ def measure(torch, gms, bench, steps, warmup, index, dist=None, dev=None, graph=
         "ms_per_step": max_ms / steps, "value": sum_traffic / max_ms / 1e6, "unit": UNIT, "bytes_per_step": bench.traffic,
         "payload_bytes": bench.payload, "phases": phases, "roofline": roofline, "clocks": sampler.summary(t0, t1),
         "gpu_launches": int(launches), "parity_ok": bool(ok), "l2": bench.config()["l2"],
+        "manifest_build_ms": getattr(bench, "build_ms", None),
     }
 
 
@@ -1165,7 +1169,7 @@ def main():
         "gpu_launches": entry["gpu_launches"], "parity_ok": entry["parity_ok"],
         "phases_ms": {k: v["mean_ms"] for k, v in entry["phases"].items()},
         "phases_ms_median_best": {k: {"median": v.get("median_ms"), "best": v.get("best_ms")} for k, v in entry["phases"].items()},
-        "geometry": gms.gms_launch_geometry(),
+        "geometry": gms.gms_launch_geometry(), "manifest_build_ms": entry.get("manifest_build_ms"),
     }
     if graphed:
         line["config"]["launch"] = f"CUDA graph replay ({bench.launches_per_step} kernel nodes per step)"

@@ -127,6 +127,9 @@ typedef struct {
  * and a few huge tensors are served by one persistent launch.
  * Block digests are laid out in entry order: tensor t owns slots
  * [first_block(t), first_block(t) + ceil(nbytes_t/4096)).
+ * The host's part is proportional to the number of tensors (validation, per-tensor
+ * positions); the chunk records themselves are written by a kernel on the device,
+ * and the call returns when they are complete (it synchronises the default stream).
  * Errors: NULL, ALIGN, RANGE, OVERLAP (destinations; overlapping sources are
  * legal), DUP_ID, NOMEM, CUDA.  nbytes == 0 is legal (no blocks, T = 0).
  * Bytes of a destination beyond nbytes are never written.
@@ -510,6 +513,8 @@ int gms_service_back_pages(gms_service *s);
  *       (defaults 1,1 / 2,1; counters 1..32, chunks 1..64)
  *   GMS_CHUNK_BLOCKS / GMS_CHUNK_BLOCKS_DIGEST         4 KiB blocks per chunk of the copy list and of the digest
  *       list (defaults 4 / 8, fewer for small manifests; 1..32)
+ *   GMS_CHECK_TABLES                                   1: gms_manifest_build reads the work lists it wrote on the
+ *       device back and compares them with a host construction of the same lists (GMS_ERR_STATE if they differ)
  */
 
 /* Launch geometry of the streaming kernels on the current device (for reporting). */

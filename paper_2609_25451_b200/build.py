@@ -15,7 +15,8 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgms.so")
-SOURCES = ["gms_api.cu", "gms_stream_kernels.cu", "gms_verify_kernels.cu", "gms_noalloc.cu", "gms_pipe.cu", "gms_service.cu"]
+SOURCES = ["gms_api.cu", "gms_stream_kernels.cu", "gms_verify_kernels.cu", "gms_build_kernels.cu", "gms_noalloc.cu", "gms_pipe.cu",
+           "gms_service.cu"]
 HEADERS = [os.path.join(CSRC, "gms_internal.h"), os.path.join(ROOT, "include", "gms.h")]
 
 

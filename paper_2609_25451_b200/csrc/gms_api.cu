@@ -20,8 +20,13 @@ using gms::Chunk;
 struct gms_manifest {
     std::vector<gms_entry> entries;
     std::vector<uint64_t> block_base;  // n + 1 prefix sums of per-tensor block counts
-    std::vector<Chunk> chunks;         // work list of the copying kernels (restore, capture)
-    std::vector<Chunk> digest_chunks;  // work list of the digest-only kernel: the same tensors cut into longer runs
+    // The two work lists live on the device, where they are also written (gms_build_kernels.cu).  Host copies are made
+    // only when something asks for them: the introspection calls, the window plan of a piecewise restore, a check.
+    uint32_t chunk_blocks = 4, digest_chunk_blocks = 8;  // 4 KiB blocks per chunk of the copy list / the digest list
+    uint64_t n_chunks = 0, n_digest_chunks = 0;
+    mutable std::vector<Chunk> chunks;         // work list of the copying kernels (restore, capture)
+    mutable std::vector<Chunk> digest_chunks;  // work list of the digest-only kernel: the same tensors cut into longer runs
+    mutable bool host_lists = false;
     uint64_t image_bytes = 0, payload = 0, n_blocks = 0;
     bool host_only = false;
     bool selftest_stall = false;  // GMS_BUILD_SELFTEST_STALL
@@ -66,24 +71,82 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Cut every tensor into runs of at most `chunk_blocks` digest blocks.  Large runs first, so that
 // the dynamic claim order ends on the small ones and the last wave of warps finishes together.
+Chunk make_chunk(const gms_manifest &m, size_t t, uint64_t off, uint64_t n)
+{
+    const gms_entry &e = m.entries[t];
+    Chunk c;
+    c.src_off = e.src_offset + off;
+    c.dst = reinterpret_cast<uint64_t>(e.dst) + off;
+    c.nbytes = (uint32_t)n;
+    c.tensor = (uint32_t)t;
+    c.gblock0 = (uint32_t)(m.block_base[t] + off / gms::kBlockBytes);
+    c.tblock0 = (uint32_t)(off / gms::kBlockBytes);
+    return c;
+}
+
+// The order is that of a stable sort by length, longest first; since all but the last chunk of a tensor have the full
+// length, it is produced directly: the full chunks in entry order, then the tensors' short last chunks sorted among
+// themselves (a list of at most one per tensor), instead of sorting a million records.
 void build_chunks(const gms_manifest &m, uint32_t chunk_blocks, std::vector<Chunk> &out)
 {
     const uint64_t chunk_bytes = (uint64_t)chunk_blocks * gms::kBlockBytes;
+    uint64_t n_full = 0, n_tail = 0;
+    for (const gms_entry &e : m.entries) {
+        n_full += e.nbytes / chunk_bytes;
+        n_tail += e.nbytes % chunk_bytes ? 1 : 0;
+    }
     out.clear();
+    out.resize(n_full + n_tail);
+    Chunk *full = out.data(), *tail = out.data() + n_full;
     for (size_t t = 0; t < m.entries.size(); ++t) {
         const gms_entry &e = m.entries[t];
         for (uint64_t off = 0; off < e.nbytes; off += chunk_bytes) {
-            Chunk c;
-            c.src_off = e.src_offset + off;
-            c.dst = reinterpret_cast<uint64_t>(e.dst) + off;
-            c.nbytes = (uint32_t)std::min<uint64_t>(chunk_bytes, e.nbytes - off);
-            c.tensor = (uint32_t)t;
-            c.gblock0 = (uint32_t)(m.block_base[t] + off / gms::kBlockBytes);
-            c.tblock0 = (uint32_t)(off / gms::kBlockBytes);
-            out.push_back(c);
+            const uint64_t n = std::min<uint64_t>(chunk_bytes, e.nbytes - off);
+            (n == chunk_bytes ? *full++ : *tail++) = make_chunk(m, t, off, n);
         }
     }
-    std::stable_sort(out.begin(), out.end(), [](const Chunk &a, const Chunk &b) { return a.nbytes > b.nbytes; });
+    std::stable_sort(out.begin() + (ptrdiff_t)n_full, out.end(), [](const Chunk &a, const Chunk &b) { return a.nbytes > b.nbytes; });
+}
+
+// Where the chunks of each tensor go in a list of the order described above: prefix sums of the full-length chunks,
+// and the position of each tensor's short last chunk (ranked by length among the short ones, longest first).
+struct ListPlan {
+    uint32_t chunk_blocks = 1;
+    uint64_t n_full = 0, n_chunks = 0;
+    std::vector<uint64_t> full_base;  // n + 1
+    std::vector<uint32_t> tail_pos;   // n; 0xffffffff: no short last chunk
+};
+
+ListPlan plan_list(const gms_manifest &m, uint32_t chunk_blocks)
+{
+    const uint64_t chunk_bytes = (uint64_t)chunk_blocks * gms::kBlockBytes;
+    const size_t n = m.entries.size();
+    ListPlan p;
+    p.chunk_blocks = chunk_blocks;
+    p.full_base.resize(n + 1);
+    p.tail_pos.assign(n, 0xffffffffu);
+    std::vector<std::pair<uint64_t, uint32_t>> tails;  // (length, tensor)
+    uint64_t acc = 0;
+    for (size_t t = 0; t < n; ++t) {
+        p.full_base[t] = acc;
+        acc += m.entries[t].nbytes / chunk_bytes;
+        if (m.entries[t].nbytes % chunk_bytes) tails.emplace_back(m.entries[t].nbytes % chunk_bytes, (uint32_t)t);
+    }
+    p.full_base[n] = p.n_full = acc;
+    std::stable_sort(tails.begin(), tails.end(), [](const auto &a, const auto &b) { return a.first > b.first; });
+    for (size_t r = 0; r < tails.size(); ++r) p.tail_pos[tails[r].second] = (uint32_t)(acc + r);
+    p.n_chunks = acc + tails.size();
+    return p;
+}
+
+// Host copies of the two lists, built on first demand (same order as the device writes them in).
+void ensure_host_lists(const gms_manifest &m)
+{
+    std::lock_guard<std::mutex> lock(m.mu);
+    if (m.host_lists) return;
+    build_chunks(m, m.chunk_blocks, m.chunks);
+    build_chunks(m, m.digest_chunk_blocks, m.digest_chunks);
+    m.host_lists = true;
 }
 
 // Tuning and test hooks read from the environment are honoured only when GMS_TUNING_HOOKS=1 is set as well, so
@@ -124,9 +187,20 @@ int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vect
 {
     if (m->host_only) return GMS_ERR_STATE;
     std::lock_guard<std::mutex> lock(m->mu);
-    if (m->by_src.empty() && !m->chunks.empty()) {
-        m->by_src = m->chunks;
-        std::stable_sort(m->by_src.begin(), m->by_src.end(), [](const Chunk &a, const Chunk &b) { return a.src_off < b.src_off; });
+    if (m->by_src.empty() && m->n_chunks) {
+        // the copy list in order of source offset.  When no two tensors share image bytes (the usual case) that is the
+        // tensors in order of their offsets, each one's chunks in order; otherwise the chunks are sorted.
+        const uint64_t chunk_bytes = (uint64_t)m->chunk_blocks * kBlockBytes;
+        std::vector<uint32_t> order(m->entries.size());
+        std::iota(order.begin(), order.end(), 0u);
+        std::stable_sort(order.begin(), order.end(),
+                         [&](uint32_t a, uint32_t b) { return m->entries[a].src_offset < m->entries[b].src_offset; });
+        m->by_src.reserve(m->n_chunks);
+        for (uint32_t t : order)
+            for (uint64_t off = 0; off < m->entries[t].nbytes; off += chunk_bytes)
+                m->by_src.push_back(make_chunk(*m, t, off, std::min<uint64_t>(chunk_bytes, m->entries[t].nbytes - off)));
+        if (!m->sources_disjoint)
+            std::stable_sort(m->by_src.begin(), m->by_src.end(), [](const Chunk &a, const Chunk &b) { return a.src_off < b.src_off; });
         cudaError_t e = cudaMalloc(&m->d_by_src, m->by_src.size() * sizeof(Chunk));
         if (e != cudaSuccess) {
             m->by_src.clear();
@@ -270,41 +344,54 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
         // work shows.  Manifests too small to give every warp two such chunks are cut finer.
         uint32_t chunk_blocks = (uint32_t)std::min<uint64_t>(4, std::max<uint64_t>(1, (n_blocks + 2ull * total_warps - 1) / (2ull * total_warps)));
         chunk_blocks = (uint32_t)env_hook("GMS_CHUNK_BLOCKS", 1, gms::kMaxChunkBlocks, chunk_blocks);
-        build_chunks(*m, chunk_blocks, m->chunks);
+        m->chunk_blocks = chunk_blocks;
         // The digest-only kernel reads twice as fast as the restore kernel moves payload and has no store side to
         // keep narrow: it is fastest on runs of 8 blocks (32 KiB) -- 2.25 ms against 2.40 ms with 4-block chunks on
         // a 16 GB manifest -- while the restore slows down on anything longer than 4.  So it gets a list of its own.
         uint32_t digest_blocks = (uint32_t)std::min<uint64_t>(8, std::max<uint64_t>(1, (n_blocks + 2ull * digest_warps - 1) / (2ull * digest_warps)));
         digest_blocks = (uint32_t)env_hook("GMS_CHUNK_BLOCKS_DIGEST", 1, gms::kMaxChunkBlocks, digest_blocks);
-        build_chunks(*m, digest_blocks, m->digest_chunks);
+        m->digest_chunk_blocks = digest_blocks;
+        const ListPlan plan = plan_list(*m, chunk_blocks), dplan = plan_list(*m, digest_blocks);
+        m->n_chunks = plan.n_chunks;
+        m->n_digest_chunks = dplan.n_chunks;
         m->n_segments = (uint32_t)((n_blocks + gms::kVerifySegBlocks - 1) / gms::kVerifySegBlocks);
 
-        // ---- device tables
+        // ---- device tables: the per-tensor columns go up in one copy, the chunk lists are written by a kernel each
         if (!m->host_only) {
             const size_t o_chunks = 0;
-            const size_t o_dchunks = align_up(o_chunks + m->chunks.size() * sizeof(Chunk), 256);
-            const size_t o_base = align_up(o_dchunks + m->digest_chunks.size() * sizeof(Chunk), 256);
+            const size_t o_dchunks = align_up(o_chunks + (size_t)m->n_chunks * sizeof(Chunk), 256);
+            const size_t o_base = align_up(o_dchunks + (size_t)m->n_digest_chunks * sizeof(Chunk), 256);
             const size_t o_ids = align_up(o_base + (n + 1) * sizeof(uint64_t), 256);
-            const size_t o_segcnt = align_up(o_ids + n * sizeof(uint64_t), 256);
+            const size_t o_src = align_up(o_ids + n * sizeof(uint64_t), 256);
+            const size_t o_dst = align_up(o_src + n * sizeof(uint64_t), 256);
+            const size_t o_len = align_up(o_dst + n * sizeof(uint64_t), 256);
+            const size_t o_fb = align_up(o_len + n * sizeof(uint64_t), 256);
+            const size_t o_dfb = align_up(o_fb + (n + 1) * sizeof(uint64_t), 256);
+            const size_t o_tp = align_up(o_dfb + (n + 1) * sizeof(uint64_t), 256);
+            const size_t o_dtp = align_up(o_tp + n * sizeof(uint32_t), 256);
+            const size_t o_segcnt = align_up(o_dtp + n * sizeof(uint32_t), 256);
             const size_t o_ctr = align_up(o_segcnt + (size_t)m->n_segments * sizeof(uint32_t), 256);
             const size_t o_status = o_ctr + (size_t)gms::kMaxCounters * gms::kCounterStride * sizeof(unsigned int);
             const size_t total = o_status + 128;
-            std::vector<uint8_t> h(total, 0);
-            if (!m->chunks.empty()) memcpy(h.data() + o_chunks, m->chunks.data(), m->chunks.size() * sizeof(Chunk));
-            if (!m->digest_chunks.empty()) memcpy(h.data() + o_dchunks, m->digest_chunks.data(), m->digest_chunks.size() * sizeof(Chunk));
-            memcpy(h.data() + o_base, m->block_base.data(), (n + 1) * sizeof(uint64_t));
-            for (size_t t = 0; t < n; ++t) memcpy(h.data() + o_ids + t * 8, &entries[t].tensor_id, 8);
+            std::vector<uint8_t> h(o_segcnt - o_base, 0);  // the columns: a few dozen bytes per tensor
+            uint8_t *hp = h.data() - o_base;                // so that hp + o_x addresses column x
+            memcpy(hp + o_base, m->block_base.data(), (n + 1) * sizeof(uint64_t));
+            for (size_t t = 0; t < n; ++t) {
+                const uint64_t dst = reinterpret_cast<uint64_t>(entries[t].dst);
+                memcpy(hp + o_ids + t * 8, &entries[t].tensor_id, 8);
+                memcpy(hp + o_src + t * 8, &entries[t].src_offset, 8);
+                memcpy(hp + o_dst + t * 8, &dst, 8);
+                memcpy(hp + o_len + t * 8, &entries[t].nbytes, 8);
+            }
+            memcpy(hp + o_fb, plan.full_base.data(), (n + 1) * sizeof(uint64_t));
+            memcpy(hp + o_dfb, dplan.full_base.data(), (n + 1) * sizeof(uint64_t));
+            if (n) memcpy(hp + o_tp, plan.tail_pos.data(), n * sizeof(uint32_t));
+            if (n) memcpy(hp + o_dtp, dplan.tail_pos.data(), n * sizeof(uint32_t));
             cudaError_t e = cudaMalloc(&m->d_tables, total);
             if (e != cudaSuccess) {
                 delete m;
                 (void)cudaGetLastError();
                 return e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : cuda_fail(e);
-            }
-            e = cudaMemcpy(m->d_tables, h.data(), total, cudaMemcpyHostToDevice);
-            if (e != cudaSuccess) {
-                cudaFree(m->d_tables);
-                delete m;
-                return cuda_fail(e);
             }
             m->d_chunks = reinterpret_cast<Chunk *>(m->d_tables + o_chunks);
             m->d_digest_chunks = reinterpret_cast<Chunk *>(m->d_tables + o_dchunks);
@@ -313,6 +400,50 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             m->d_seg_count = reinterpret_cast<uint32_t *>(m->d_tables + o_segcnt);
             m->d_counter = reinterpret_cast<unsigned int *>(m->d_tables + o_ctr);
             m->d_status = reinterpret_cast<unsigned long long *>(m->d_tables + o_status);
+            e = cudaMemcpy(m->d_tables + o_base, h.data(), h.size(), cudaMemcpyHostToDevice);
+            if (e == cudaSuccess) e = cudaMemset(m->d_tables + o_segcnt, 0, total - o_segcnt);
+            gms::ExpandArgs x;
+            x.src_offset = reinterpret_cast<const uint64_t *>(m->d_tables + o_src);
+            x.dst = reinterpret_cast<const uint64_t *>(m->d_tables + o_dst);
+            x.nbytes = reinterpret_cast<const uint64_t *>(m->d_tables + o_len);
+            x.block_base = m->d_block_base;
+            x.n_tensors = (uint32_t)n;
+            x.full_base = reinterpret_cast<const uint64_t *>(m->d_tables + o_fb);
+            x.tail_pos = reinterpret_cast<const uint32_t *>(m->d_tables + o_tp);
+            x.n_full = plan.n_full;
+            x.chunk_blocks = chunk_blocks;
+            x.out = m->d_chunks;
+            if (e == cudaSuccess) e = gms::launch_expand_chunks(x, nullptr);
+            x.full_base = reinterpret_cast<const uint64_t *>(m->d_tables + o_dfb);
+            x.tail_pos = reinterpret_cast<const uint32_t *>(m->d_tables + o_dtp);
+            x.n_full = dplan.n_full;
+            x.chunk_blocks = digest_blocks;
+            x.out = m->d_digest_chunks;
+            if (e == cudaSuccess) e = gms::launch_expand_chunks(x, nullptr);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(nullptr);  // the lists are complete when the call returns
+            if (e == cudaSuccess && env_hook("GMS_CHECK_TABLES", 0, 1, 0)) {
+                // test hook: the device-written lists must equal the host's construction of the same order
+                ensure_host_lists(*m);
+                std::vector<Chunk> got(m->n_chunks + m->n_digest_chunks);
+                e = cudaMemcpy(got.data(), m->d_chunks, (size_t)m->n_chunks * sizeof(Chunk), cudaMemcpyDeviceToHost);
+                if (e == cudaSuccess)
+                    e = cudaMemcpy(got.data() + m->n_chunks, m->d_digest_chunks, (size_t)m->n_digest_chunks * sizeof(Chunk),
+                                   cudaMemcpyDeviceToHost);
+                const bool same = e == cudaSuccess && m->chunks.size() == m->n_chunks && m->digest_chunks.size() == m->n_digest_chunks &&
+                                  (m->n_chunks == 0 || memcmp(got.data(), m->chunks.data(), (size_t)m->n_chunks * sizeof(Chunk)) == 0) &&
+                                  (m->n_digest_chunks == 0 || memcmp(got.data() + m->n_chunks, m->digest_chunks.data(),
+                                                                     (size_t)m->n_digest_chunks * sizeof(Chunk)) == 0);
+                if (e == cudaSuccess && !same) {
+                    cudaFree(m->d_tables);
+                    delete m;
+                    return GMS_ERR_STATE;
+                }
+            }
+            if (e != cudaSuccess) {
+                cudaFree(m->d_tables);
+                delete m;
+                return cuda_fail(e);
+            }
         }
         *out = m;
         return GMS_OK;
@@ -356,14 +487,19 @@ int gms_manifest_block_base(const gms_manifest *m, size_t entry_index, uint64_t 
 int gms_manifest_chunk_count(const gms_manifest *m, uint64_t *n_chunks)
 {
     if (!m || !n_chunks) return GMS_ERR_NULL;
-    *n_chunks = m->chunks.size();
+    *n_chunks = m->n_chunks;
     return GMS_OK;
 }
 
 int gms_manifest_chunk(const gms_manifest *m, uint64_t i, uint64_t *entry_index, uint64_t *tensor_byte_offset, uint64_t *nbytes)
 {
     if (!m) return GMS_ERR_NULL;
-    if (i >= m->chunks.size()) return GMS_ERR_ARG;
+    if (i >= m->n_chunks) return GMS_ERR_ARG;
+    try {
+        ensure_host_lists(*m);
+    } catch (const std::bad_alloc &) {
+        return GMS_ERR_NOMEM;
+    }
     const Chunk &c = m->chunks[i];
     if (entry_index) *entry_index = c.tensor;
     if (tensor_byte_offset) *tensor_byte_offset = (uint64_t)c.tblock0 * gms::kBlockBytes;
@@ -392,7 +528,7 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
 {
     gms::StreamArgs a;
     a.chunks = store ? m->d_chunks : m->d_digest_chunks;
-    a.n_chunks = (uint32_t)(store ? m->chunks.size() : m->digest_chunks.size());
+    a.n_chunks = (uint32_t)(store ? m->n_chunks : m->n_digest_chunks);
     a.image = static_cast<const uint8_t *>(image);
     a.block_digests = d_block_digests;
     a.tensor_digests = d_tensor_digests;

@@ -105,6 +105,21 @@ cudaError_t launch_verify_counted(const VerifyArgs &a, cudaStream_t s);
 cudaError_t launch_verify_tensor_counts(const VerifyArgs &a, uint32_t *counts, cudaStream_t s);
 cudaError_t launch_copy_u64(uint64_t *dst, const uint64_t *src, uint64_t n, cudaStream_t s);
 
+// Expansion of the layout record into one chunk list on the device (gms_build_kernels.cu).  All pointers are device
+// memory; the per-tensor columns are the record's fields, full_base the prefix sums of full-length chunks per tensor,
+// tail_pos the list position of each tensor's short last chunk (0xffffffff: it has none).
+struct ExpandArgs {
+    const uint64_t *src_offset, *dst, *nbytes;  // n_tensors each
+    const uint64_t *block_base;                 // n_tensors + 1
+    const uint64_t *full_base;                  // n_tensors + 1
+    const uint32_t *tail_pos;                   // n_tensors
+    uint32_t n_tensors;
+    uint64_t n_full;
+    uint32_t chunk_blocks;
+    Chunk *out;
+};
+cudaError_t launch_expand_chunks(const ExpandArgs &a, cudaStream_t s);
+
 // A window of a restore that is fed piecewise (file -> pinned buffer -> device): a run of the
 // chunk list sorted by source offset whose sources all lie in image bytes [src_lo, src_hi).
 struct SrcWindow {

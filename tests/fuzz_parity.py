@@ -44,6 +44,7 @@ def random_sizes(rng):
 def one_manifest_round(rng, it):
     sizes = random_sizes(rng)
     os.environ["GMS_TUNING_HOOKS"] = "1"  # the hooks below are ignored without it
+    os.environ["GMS_CHECK_TABLES"] = "1"  # device-written work lists are compared with the host's construction
     os.environ["GMS_CHUNK_BLOCKS"] = str(int(rng.choice([1, 2, 3, 4, 4, 4, 7, 16, 32])))
     os.environ["GMS_CHUNK_BLOCKS_DIGEST"] = str(int(rng.choice([1, 3, 8, 8, 8, 5, 16, 32])))
     w = W.pack_layout(f"fuzz{it}", sizes, seed=int(rng.integers(1 << 30)), guard=int(rng.choice([16, 64, 256])))

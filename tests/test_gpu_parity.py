@@ -310,6 +310,29 @@ def test_kv_restore_other_block_sizes_and_host_source(oracle):
     run_kv(oracle, 5, 50, 32768, np.zeros(0, np.int32), 0, 95)
 
 
+def test_device_written_work_lists_equal_the_hosts(monkeypatch):
+    """gms_manifest_build writes the chunk records on the device; with the check hook on it reads them back and
+    compares them with the host's construction of the same order (a difference would make the build fail).  The
+    introspection calls, which use the host's lists, must describe a partition of every tensor."""
+    monkeypatch.setenv("GMS_TUNING_HOOKS", "1")
+    monkeypatch.setenv("GMS_CHECK_TABLES", "1")
+    for w in (W.pack_layout("edge", EDGE_SIZES, seed=11), W.mixed_manifest(n_small=3000, n_large=2, large_bytes=(8 << 20) + 24, round16=False),
+              W.llama3_8b_manifest(shrink=8), W.pack_layout("empty", [0, 0], seed=1)):
+        for blocks in ("1", "4", "7", "32"):
+            monkeypatch.setenv("GMS_CHUNK_BLOCKS", blocks)
+            monkeypatch.setenv("GMS_CHUNK_BLOCKS_DIGEST", str(33 - int(blocks)))
+            d = DeviceWorkload(w, np.zeros(w.image_bytes, np.uint8))  # the build itself is the check
+            covered = {}
+            for i in range(gms.gms_manifest_chunk_count(d.m)):
+                t, off, n = gms.gms_manifest_chunk(d.m, i)
+                covered.setdefault(t, []).append((off, n))
+            for t, r in enumerate(w.rows):
+                pieces = sorted(covered.get(t, []))
+                assert sum(n for _, n in pieces) == int(r["nbytes"])
+                assert all(pieces[k][0] + pieces[k][1] == pieces[k + 1][0] for k in range(len(pieces) - 1))
+            d.close()
+
+
 def test_geometry_is_a_multiple_of_the_sm_count():
     g = gms.gms_launch_geometry()
     sms = torch.cuda.get_device_properties(0).multi_processor_count

@@ -35,6 +35,7 @@ def test_parity_in_other_launch_shapes(env):
     full = dict(os.environ)
     full.update(env)
     full["GMS_TUNING_HOOKS"] = "1"  # the library ignores the shape hooks without it
+    full["GMS_CHECK_TABLES"] = "1"  # every manifest built in the child compares its device-written work lists with the host's
     r = subprocess.run([sys.executable, os.path.join(HERE, "geometry_check.py")], env=full, capture_output=True, text=True,
                        timeout=600)
     assert r.returncode == 0 and r.stdout.strip().startswith("OK"), r.stdout[-2000:] + r.stderr[-4000:]
