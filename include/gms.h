@@ -385,9 +385,10 @@ int gms_host_image_free(void *host_ptr);
  * scattered + digested from there by the restore kernel while the next one is read.  If the device
  * buffers cannot be allocated the pipe still works: the kernel then reads the pinned buffers across
  * the host link itself, which reaches about 93 % of what the copy engine does.
- * The first gms_restore_fd (or gms_restore_staged) on a manifest builds and uploads a copy of its work list
- * sorted by source offset: that call allocates device memory and synchronises, so it must not be made
- * while a stream capture is in progress.
+ * The first gms_restore_fd (or gms_restore_staged) on a manifest writes a copy of its work list sorted by
+ * source offset (on the device, like the other lists) and plans the windows; that call allocates device
+ * memory and synchronises, so it must not be made while a stream capture is in progress.  Later calls
+ * with the same buffer size reuse the plan.
  * gms_restore_fd is synchronous: on return the stream has been synchronised and the outputs hold
  * exactly what gms_restore would have produced from the same bytes (image byte k = file byte
  * file_offset + k).  One restore at a time per pipe.  Errors: NULL, ARG (bad sizes; a chunk larger

@@ -6,6 +6,7 @@
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
 #include <numeric>
@@ -42,10 +43,12 @@ struct gms_manifest {
     uint64_t *d_expected = nullptr;
     bool has_expected = false;
     uint32_t n_segments = 0;
-    // chunk list sorted by source offset, for restores fed window by window (built on first use)
+    // chunk list sorted by source offset, for restores fed window by window (built on first use), and the window
+    // plans made from it so far, by buffer size
     mutable std::mutex mu;
-    mutable std::vector<Chunk> by_src;
     mutable Chunk *d_by_src = nullptr;
+    mutable std::map<uint64_t, std::vector<gms::SrcWindow>> window_plans;
+    const uint64_t *d_src = nullptr, *d_dst = nullptr, *d_len = nullptr;  // the record's columns on the device
 };
 
 namespace {
@@ -187,51 +190,117 @@ int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vect
 {
     if (m->host_only) return GMS_ERR_STATE;
     std::lock_guard<std::mutex> lock(m->mu);
-    if (m->by_src.empty() && m->n_chunks) {
-        // the copy list in order of source offset.  When no two tensors share image bytes (the usual case) that is the
-        // tensors in order of their offsets, each one's chunks in order; otherwise the chunks are sorted.
-        const uint64_t chunk_bytes = (uint64_t)m->chunk_blocks * kBlockBytes;
-        std::vector<uint32_t> order(m->entries.size());
-        std::iota(order.begin(), order.end(), 0u);
-        std::stable_sort(order.begin(), order.end(),
-                         [&](uint32_t a, uint32_t b) { return m->entries[a].src_offset < m->entries[b].src_offset; });
-        m->by_src.reserve(m->n_chunks);
+    {
+        auto cached = m->window_plans.find(buffer_bytes);  // planned before (the sorted list is on the device by then)
+        if (cached != m->window_plans.end()) {
+            *out = cached->second;
+            return GMS_OK;
+        }
+    }
+    const size_t n = m->entries.size();
+    const uint64_t chunk_bytes = (uint64_t)m->chunk_blocks * kBlockBytes;
+    // the copy list in order of source offset: the tensors in order of their offsets, each one's chunks in order
+    std::vector<uint32_t> order(n);
+    std::iota(order.begin(), order.end(), 0u);
+    std::stable_sort(order.begin(), order.end(),
+                     [&](uint32_t a, uint32_t b) { return m->entries[a].src_offset < m->entries[b].src_offset; });
+    std::vector<Chunk> sorted;  // only when tensors share image bytes: then the chunks themselves have to be sorted
+    if (!m->sources_disjoint) {
+        sorted.reserve(m->n_chunks);
         for (uint32_t t : order)
             for (uint64_t off = 0; off < m->entries[t].nbytes; off += chunk_bytes)
-                m->by_src.push_back(make_chunk(*m, t, off, std::min<uint64_t>(chunk_bytes, m->entries[t].nbytes - off)));
-        if (!m->sources_disjoint)
-            std::stable_sort(m->by_src.begin(), m->by_src.end(), [](const Chunk &a, const Chunk &b) { return a.src_off < b.src_off; });
-        cudaError_t e = cudaMalloc(&m->d_by_src, m->by_src.size() * sizeof(Chunk));
+                sorted.push_back(make_chunk(*m, t, off, std::min<uint64_t>(chunk_bytes, m->entries[t].nbytes - off)));
+        std::stable_sort(sorted.begin(), sorted.end(), [](const Chunk &a, const Chunk &b) { return a.src_off < b.src_off; });
+    }
+    if (!m->d_by_src && m->n_chunks) {
+        cudaError_t e = cudaMalloc(&m->d_by_src, (size_t)m->n_chunks * sizeof(Chunk));
         if (e != cudaSuccess) {
-            m->by_src.clear();
             (void)cudaGetLastError();
             return e == cudaErrorMemoryAllocation ? GMS_ERR_NOMEM : cuda_fail(e);
         }
-        e = cudaMemcpy(m->d_by_src, m->by_src.data(), m->by_src.size() * sizeof(Chunk), cudaMemcpyHostToDevice);
+        if (m->sources_disjoint) {
+            // written on the device like the other lists: every tensor's chunks, its short last one included, in place
+            std::vector<uint64_t> base(n + 1);
+            uint64_t acc = 0;
+            for (size_t k = 0; k < n; ++k) {
+                base[k] = acc;
+                acc += (m->entries[order[k]].nbytes + chunk_bytes - 1) / chunk_bytes;
+            }
+            base[n] = acc;
+            const size_t o_perm = (n + 1) * sizeof(uint64_t), o_tail = o_perm + n * sizeof(uint32_t), bytes = o_tail + n * sizeof(uint32_t);
+            std::vector<uint8_t> h(bytes, 0xff);  // tail positions: all "none"
+            memcpy(h.data(), base.data(), (n + 1) * sizeof(uint64_t));
+            if (n) memcpy(h.data() + o_perm, order.data(), n * sizeof(uint32_t));
+            uint8_t *tmp = nullptr;
+            e = cudaMalloc(&tmp, bytes);
+            if (e == cudaSuccess) e = cudaMemcpy(tmp, h.data(), bytes, cudaMemcpyHostToDevice);
+            ExpandArgs x;
+            x.src_offset = m->d_src;
+            x.dst = m->d_dst;
+            x.nbytes = m->d_len;
+            x.block_base = m->d_block_base;
+            x.full_base = reinterpret_cast<const uint64_t *>(tmp);
+            x.perm = reinterpret_cast<const uint32_t *>(tmp + o_perm);
+            x.tail_pos = reinterpret_cast<const uint32_t *>(tmp + o_tail);
+            x.n_tensors = (uint32_t)n;
+            x.n_full = acc;
+            x.chunk_blocks = m->chunk_blocks;
+            x.out = m->d_by_src;
+            if (e == cudaSuccess) e = launch_expand_chunks(x, nullptr);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(nullptr);
+            if (tmp) cudaFree(tmp);
+        } else {
+            e = cudaMemcpy(m->d_by_src, sorted.data(), sorted.size() * sizeof(Chunk), cudaMemcpyHostToDevice);
+        }
         if (e != cudaSuccess) {
             cudaFree(m->d_by_src);
             m->d_by_src = nullptr;
-            m->by_src.clear();
             return cuda_fail(e);
         }
     }
+    // greedy cut: a window takes chunks, in list order, while their sources span at most one buffer
     out->clear();
-    size_t i = 0;
-    while (i < m->by_src.size()) {
+    size_t ti = 0;          // cursor: tensor slot in `order` ...
+    uint64_t off = 0;       // ... and byte offset of the next chunk inside it (disjoint sources), or
+    size_t si = 0;          // index into `sorted` (shared sources)
+    auto skip_empty = [&] {
+        while (ti < n && off >= m->entries[order[ti]].nbytes) ++ti, off = 0;
+    };
+    skip_empty();
+    uint64_t i = 0;
+    while (i < m->n_chunks) {
         SrcWindow w;
         w.first_chunk = (uint32_t)i;
-        w.src_lo = m->by_src[i].src_off;
-        w.src_hi = w.src_lo;
-        while (i < m->by_src.size()) {
-            const uint64_t end = m->by_src[i].src_off + m->by_src[i].nbytes;
+        const uint64_t first = i;
+        bool started = false;
+        w.src_lo = w.src_hi = 0;
+        while (i < m->n_chunks) {
+            uint64_t src, len;
+            if (m->sources_disjoint) {
+                const gms_entry &e = m->entries[order[ti]];
+                src = e.src_offset + off;
+                len = std::min<uint64_t>(chunk_bytes, e.nbytes - off);
+            } else {
+                src = sorted[si].src_off;
+                len = sorted[si].nbytes;
+            }
+            if (!started) w.src_lo = w.src_hi = src, started = true;
+            const uint64_t end = src + len;
             if (std::max(end, w.src_hi) - w.src_lo > buffer_bytes) break;
             w.src_hi = std::max(end, w.src_hi);
             ++i;
+            if (m->sources_disjoint) {
+                off += chunk_bytes;
+                skip_empty();
+            } else {
+                ++si;
+            }
         }
-        if (i == w.first_chunk) return GMS_ERR_ARG;  // a single chunk does not fit the buffer
-        w.n_chunks = (uint32_t)(i - w.first_chunk);
+        if (i == first) return GMS_ERR_ARG;  // a single chunk does not fit the buffer
+        w.n_chunks = (uint32_t)(i - first);
         out->push_back(w);
     }
+    m->window_plans[buffer_bytes] = *out;
     return GMS_OK;
 }
 
@@ -403,9 +472,10 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             e = cudaMemcpy(m->d_tables + o_base, h.data(), h.size(), cudaMemcpyHostToDevice);
             if (e == cudaSuccess) e = cudaMemset(m->d_tables + o_segcnt, 0, total - o_segcnt);
             gms::ExpandArgs x;
-            x.src_offset = reinterpret_cast<const uint64_t *>(m->d_tables + o_src);
-            x.dst = reinterpret_cast<const uint64_t *>(m->d_tables + o_dst);
-            x.nbytes = reinterpret_cast<const uint64_t *>(m->d_tables + o_len);
+            x.src_offset = m->d_src = reinterpret_cast<const uint64_t *>(m->d_tables + o_src);
+            x.dst = m->d_dst = reinterpret_cast<const uint64_t *>(m->d_tables + o_dst);
+            x.nbytes = m->d_len = reinterpret_cast<const uint64_t *>(m->d_tables + o_len);
+            x.perm = nullptr;
             x.block_base = m->d_block_base;
             x.n_tensors = (uint32_t)n;
             x.full_base = reinterpret_cast<const uint64_t *>(m->d_tables + o_fb);

@@ -13,7 +13,7 @@ __global__ void gms_expand_chunks_kernel(ExpandArgs a)
     const uint64_t chunk_bytes = (uint64_t)a.chunk_blocks * kBlockBytes;
     const uint64_t total = a.n_full + a.n_tensors, step = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += step) {
-        uint32_t t;
+        uint32_t t;  // slot of the tensor in the list's tensor order
         uint64_t off, pos;
         if (i < a.n_full) {
             // tensor t with full_base[t] <= i < full_base[t + 1] (tensors without a full chunk share a base)
@@ -31,13 +31,14 @@ __global__ void gms_expand_chunks_kernel(ExpandArgs a)
             off = (a.full_base[t + 1] - a.full_base[t]) * chunk_bytes;
             pos = a.tail_pos[t];
         }
-        const uint64_t nbytes = a.nbytes[t];
+        const uint32_t e = a.perm ? a.perm[t] : t;  // the entry
+        const uint64_t nbytes = a.nbytes[e];
         Chunk c;
-        c.src_off = a.src_offset[t] + off;
-        c.dst = a.dst[t] + off;
+        c.src_off = a.src_offset[e] + off;
+        c.dst = a.dst[e] + off;
         c.nbytes = (uint32_t)(nbytes - off < chunk_bytes ? nbytes - off : chunk_bytes);
-        c.tensor = t;
-        c.gblock0 = (uint32_t)(a.block_base[t] + off / kBlockBytes);
+        c.tensor = e;
+        c.gblock0 = (uint32_t)(a.block_base[e] + off / kBlockBytes);
         c.tblock0 = (uint32_t)(off / kBlockBytes);
         a.out[pos] = c;
     }

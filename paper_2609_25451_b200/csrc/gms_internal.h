@@ -113,6 +113,8 @@ struct ExpandArgs {
     const uint64_t *block_base;                 // n_tensors + 1
     const uint64_t *full_base;                  // n_tensors + 1
     const uint32_t *tail_pos;                   // n_tensors
+    const uint32_t *perm;                       // null, or n_tensors: list slot -> entry index (lists in another tensor order;
+                                                // full_base and tail_pos are then indexed by slot, the columns by entry)
     uint32_t n_tensors;
     uint64_t n_full;
     uint32_t chunk_blocks;

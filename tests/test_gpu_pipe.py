@@ -107,6 +107,49 @@ def test_restore_staged_equals_restore_of_the_same_bytes(oracle, n_buffers, buff
         gms.gms_host_image_free(hptr)
 
 
+@pytest.mark.gpu
+def test_piecewise_restores_with_tensors_that_share_image_bytes(oracle, tmp_path):
+    """Overlapping sources are legal for a restore (several tensors filled from the same image bytes).  The window
+    plan then has to sort chunks of different tensors among each other; both piecewise restores must still give the
+    oracle's bytes and digests."""
+    from gpu_harness import payload_of
+
+    w = W.pack_layout("shared", [(3 << 20) + 40, 70000, 5 << 20, 4096, 1 << 20], seed=9)
+    w.rows["src_offset"][2] = w.rows["src_offset"][0] + 65536   # tensor 2 starts inside tensor 0 and runs past its end
+    w.rows["src_offset"][3] = w.rows["src_offset"][1]           # tensor 3 is the head of tensor 1
+    image = W.random_bytes_host(w.image_bytes, seed=79)
+    slab_h = np.full(w.slab_bytes, FILL, np.uint8)
+    rc, obd, otd = oracle.restore(oracle_record(oracle, w), image, slab_h)
+    assert rc == 0
+    d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    hptr, _, arr = gms.gms_host_image_alloc(w.image_bytes)
+    arr[:] = image
+    path = str(tmp_path / "shared.bin")
+    _write_image(path, image, 0)
+    stage = gms.gms_stage_create(2, 1 << 20)
+    pipe = gms.gms_pipe_create(2, 1 << 20, 3)
+    fd = os.open(path, os.O_RDONLY)
+    try:
+        for how in ("staged", "fd", "staged"):
+            d.slab.fill_(FILL)
+            d.reset_outputs()
+            if how == "staged":
+                gms.gms_restore_staged(d.m, stage, hptr, d.bd_ptr(), d.td_ptr())
+            else:
+                gms.gms_restore_fd(d.m, pipe, fd, 0, d.bd_ptr(), d.td_ptr())
+            torch.cuda.synchronize()
+            assert gms.gms_last_device_status(d.m) == 0
+            assert np.array_equal(d.slab_host(), slab_h), how
+            assert np.array_equal(payload_of(d.bd, d.nb), obd) and np.array_equal(payload_of(d.td, d.nt), otd), how
+    finally:
+        os.close(fd)
+        torch.cuda.synchronize()
+        pipe.close()
+        stage.close()
+        d.close()
+        gms.gms_host_image_free(hptr)
+
+
 def test_stage_argument_checks_need_no_gpu():
     out = ctypes.c_void_p()
     L = gms.lib()
