@@ -491,6 +491,9 @@ def measure(torch, gms, bench, steps, warmup, index, dist=None, dev=None, graph=
         ratio = NCU_DRAM_BYTES_PER_PAYLOAD_BYTE.get(dom)
         roofline = {"kernel": bench.kernel_text(), "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_datasheet_8TBps": achieved / DATASHEET_HBM_GBS,
+                    "achieved_median": bench.phase_bytes[dom] / stats[dom]["median"] / 1e6,
+                    "frac_median": bench.phase_bytes[dom] / stats[dom]["median"] / 1e6 / peak,
+                    "duration_ms": {"mean": stats[dom]["mean"], "median": stats[dom]["median"], "best": stats[dom]["best"]},
                     "algorithmic_bytes_per_launch": bench.phase_bytes[dom], "traffic": (ratio * bench.payload) if ratio else None,
                     "traffic_source": NCU_TRAFFIC_SOURCE if ratio else None}
     return {
