@@ -379,6 +379,7 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
     uint32_t is = 0;               // ring slot of the next block to issue   (issued % S)
     uint32_t cs = 0, cparity = 0;  // ring slot and barrier phase of the next block to digest
     uint32_t my_lo = 0, my_hi = 0;
+    uint64_t want = 0;  // fused compare: the recorded digest of the block whose digest this lane holds
     // share of a tensor digest gathered over consecutive chunks of the same tensor: one atomic per run, not per chunk
     uint32_t run_tensor = 0xffffffffu;
     uint64_t run_val = 0;
@@ -452,6 +453,9 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
             c_tblock0 = r1.y;
             c_blocks = (c_nbytes + kBlockBytes - 1) >> 12;
             c_next = 0;
+            // fused compare: the recorded digests of this chunk's blocks are fetched now and used at its end, so that
+            // their latency lies under the chunk's digest work instead of behind it
+            if (expected && lane < c_blocks) want = __ldg(expected + c_gblock0 + lane);
         }
         const uint8_t *stage = ring + s * kBlockBytes;
         if (kStore && lane == 0) {
@@ -479,7 +483,7 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
             if (lane < c_blocks) {
                 const uint64_t raw = ((uint64_t)my_hi << 32) | my_lo, myD = raw ^ (raw >> 31);
                 if (block_digests) block_digests[(uint64_t)c_gblock0 + lane] = myD;
-                if (expected && __ldg(expected + c_gblock0 + lane) != myD) atomicAdd(seg_count + ((c_gblock0 + lane) >> kVerifySegShift), 1u);
+                if (expected && want != myD) atomicAdd(seg_count + ((c_gblock0 + lane) >> kVerifySegShift), 1u);
                 t = mix_full32(myD ^ ((uint64_t)(c_tblock0 + lane) * kG));
             }
             t = warp_xor64(t);
