@@ -333,6 +333,37 @@ def test_device_written_work_lists_equal_the_hosts(monkeypatch):
             d.close()
 
 
+def test_thirty_thousand_small_tensors_and_exact_chunk_multiples(oracle):
+    """Many tensors, most of them shorter than one chunk (so nearly every chunk is some tensor's short last one and
+    the list order is decided by the ranking of those), next to tensors that are exact multiples of the chunk
+    lengths (no short chunk at all) and empty ones: bytes, digests, fused verify against the oracle."""
+    rng = np.random.default_rng(123)
+    sizes = [int(x) for x in rng.integers(0, 9000, 30000)]
+    sizes[::97] = [0] * len(sizes[::97])
+    sizes += [16384 * 3, 32768 * 5, 16384, 32768, 4096, 65536 * 7]
+    w = W.pack_layout("many-small", sizes, seed=31, guard=16)
+    image = W.random_bytes_host(w.image_bytes, seed=32)
+    want_slab, want_bd, want_td = oracle_restore(oracle, w, image)
+    d = DeviceWorkload(w, image)
+    bd, td = d.restore()
+    assert np.array_equal(d.slab_host(), want_slab) and np.array_equal(bd, want_bd) and np.array_equal(td, want_td)
+    bd2, td2 = d.digest()
+    assert np.array_equal(bd2, want_bd) and np.array_equal(td2, want_td)
+    gms.gms_manifest_set_expected(d.m, d.bd_ptr())
+    rec = oracle_record(oracle, w)
+    flips = W.flip_positions(w, 40, seed=33)
+    for row, byte, bit in flips:
+        d.flip(row, byte, bit)
+        want_slab[int(w.rows[row]["dst_offset"]) + byte] ^= 1 << bit
+    _, obd, otd = oracle.digest(rec, want_slab)
+    ocount, omm = oracle.verify(rec, obd, want_bd, cap=64)
+    fbd, ftd, count, pairs = d.fused(64)
+    assert np.array_equal(fbd, obd) and np.array_equal(ftd, otd)
+    assert count == ocount == 40 and pairs == [(int(m["tensor_id"]), int(m["block"])) for m in omm]
+    assert d.verify(cap=64) == (count, pairs)
+    d.close()
+
+
 def test_geometry_is_a_multiple_of_the_sm_count():
     g = gms.gms_launch_geometry()
     sms = torch.cuda.get_device_properties(0).multi_processor_count
