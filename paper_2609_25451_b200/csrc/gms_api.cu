@@ -72,6 +72,30 @@ uint64_t blocks_of(uint64_t nbytes) { return nbytes / gms::kBlockBytes + (nbytes
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Stable sort of (key, payload) pairs by key.  Validation and list planning sort the tensors' ids, destination and
+// source ranges and short-chunk lengths; with tens of thousands of tensors a comparison sort is then most of the
+// host's build time, so from a few thousand pairs on this is an LSD radix sort, 11 bits at a time, that skips the
+// digits in which all keys agree.
+void radix_sort_pairs(std::vector<std::pair<uint64_t, uint64_t>> &v)
+{
+    if (v.size() < 2048) {
+        std::stable_sort(v.begin(), v.end(), [](const auto &a, const auto &b) { return a.first < b.first; });
+        return;
+    }
+    uint64_t all_or = 0, all_and = ~0ull;
+    for (const auto &p : v) all_or |= p.first, all_and &= p.first;
+    std::vector<std::pair<uint64_t, uint64_t>> tmp(v.size());
+    uint32_t count[2049];
+    for (int shift = 0; shift < 64; shift += 11) {
+        if ((((all_or ^ all_and) >> shift) & 0x7ffu) == 0) continue;  // this digit does not vary
+        memset(count, 0, sizeof count);
+        for (const auto &p : v) ++count[((p.first >> shift) & 0x7ffu) + 1];
+        for (size_t d = 0; d < 2048; ++d) count[d + 1] += count[d];
+        for (const auto &p : v) tmp[count[(p.first >> shift) & 0x7ffu]++] = p;
+        v.swap(tmp);
+    }
+}
+
 // Cut every tensor into runs of at most `chunk_blocks` digest blocks.  Large runs first, so that
 // the dynamic claim order ends on the small ones and the last wave of warps finishes together.
 Chunk make_chunk(const gms_manifest &m, size_t t, uint64_t off, uint64_t n)
@@ -128,15 +152,17 @@ ListPlan plan_list(const gms_manifest &m, uint32_t chunk_blocks)
     p.chunk_blocks = chunk_blocks;
     p.full_base.resize(n + 1);
     p.tail_pos.assign(n, 0xffffffffu);
-    std::vector<std::pair<uint64_t, uint32_t>> tails;  // (length, tensor)
+    // short last chunks ranked by length, longest first, entry order among equals: lengths are below 128 KiB, so the
+    // key (chunk_bytes - length) is sorted ascending by the stable radix sort
+    std::vector<std::pair<uint64_t, uint64_t>> tails;  // (chunk_bytes - length, tensor)
     uint64_t acc = 0;
     for (size_t t = 0; t < n; ++t) {
         p.full_base[t] = acc;
         acc += m.entries[t].nbytes / chunk_bytes;
-        if (m.entries[t].nbytes % chunk_bytes) tails.emplace_back(m.entries[t].nbytes % chunk_bytes, (uint32_t)t);
+        if (m.entries[t].nbytes % chunk_bytes) tails.emplace_back(chunk_bytes - m.entries[t].nbytes % chunk_bytes, t);
     }
     p.full_base[n] = p.n_full = acc;
-    std::stable_sort(tails.begin(), tails.end(), [](const auto &a, const auto &b) { return a.first > b.first; });
+    radix_sort_pairs(tails);
     for (size_t r = 0; r < tails.size(); ++r) p.tail_pos[tails[r].second] = (uint32_t)(acc + r);
     p.n_chunks = acc + tails.size();
     return p;
@@ -353,27 +379,30 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
     }
     gms_manifest *m = nullptr;
     try {
-        std::vector<uint32_t> order(n);
-        std::iota(order.begin(), order.end(), 0u);
-        std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return entries[a].tensor_id < entries[b].tensor_id; });
+        // the three checks sort plain key arrays (ids; (start, end) of destinations; (start, end) of sources): with ten
+        // thousand tensors that is a few hundred microseconds each, where sorting indices into the records took over a
+        // millisecond each
+        std::vector<std::pair<uint64_t, uint64_t>> span(n);
+        for (size_t t = 0; t < n; ++t) span[t] = {entries[t].tensor_id, 0};
+        radix_sort_pairs(span);
         for (size_t i = 1; i < n; ++i)
-            if (entries[order[i]].tensor_id == entries[order[i - 1]].tensor_id) return GMS_ERR_DUP_ID;
-        // destinations pairwise disjoint: sort the non-empty ones by address, compare neighbours
-        std::vector<uint32_t> live;
-        for (uint32_t t = 0; t < n; ++t)
-            if (entries[t].nbytes) live.push_back(t);
-        std::sort(live.begin(), live.end(), [&](uint32_t a, uint32_t b) {
-            return reinterpret_cast<uint64_t>(entries[a].dst) < reinterpret_cast<uint64_t>(entries[b].dst);
-        });
-        for (size_t i = 1; i < live.size(); ++i) {
-            const gms_entry &p = entries[live[i - 1]], &q = entries[live[i]];
-            if (reinterpret_cast<uint64_t>(p.dst) + p.nbytes > reinterpret_cast<uint64_t>(q.dst)) return GMS_ERR_OVERLAP;
-        }
+            if (span[i].first == span[i - 1].first) return GMS_ERR_DUP_ID;
+        // destinations pairwise disjoint: sort the non-empty ones by address, compare neighbours (with equal starts
+        // any order will do: two non-empty ranges that start together overlap)
+        span.clear();
+        for (size_t t = 0; t < n; ++t)
+            if (entries[t].nbytes) span.emplace_back(reinterpret_cast<uint64_t>(entries[t].dst), reinterpret_cast<uint64_t>(entries[t].dst) + entries[t].nbytes);
+        radix_sort_pairs(span);
+        for (size_t i = 1; i < span.size(); ++i)
+            if (span[i - 1].second > span[i].first) return GMS_ERR_OVERLAP;
 
         bool sources_disjoint = true;
-        std::sort(live.begin(), live.end(), [&](uint32_t a, uint32_t b) { return entries[a].src_offset < entries[b].src_offset; });
-        for (size_t i = 1; i < live.size(); ++i)
-            if (entries[live[i - 1]].src_offset + entries[live[i - 1]].nbytes > entries[live[i]].src_offset) sources_disjoint = false;
+        span.clear();
+        for (size_t t = 0; t < n; ++t)
+            if (entries[t].nbytes) span.emplace_back(entries[t].src_offset, entries[t].src_offset + entries[t].nbytes);
+        radix_sort_pairs(span);
+        for (size_t i = 1; i < span.size(); ++i)
+            if (span[i - 1].second > span[i].first) sources_disjoint = false;
 
         m = new gms_manifest();
         m->sources_disjoint = sources_disjoint;
