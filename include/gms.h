@@ -129,7 +129,8 @@ typedef struct {
  * [first_block(t), first_block(t) + ceil(nbytes_t/4096)).
  * The host's part is proportional to the number of tensors (validation, per-tensor
  * positions); the chunk records themselves are written by a kernel on the device,
- * and the call returns when they are complete (it synchronises the default stream).
+ * on a stream of the library's own, and the call returns when they are complete
+ * (it does not wait for work the caller has queued on other streams).
  * Errors: NULL, ALIGN, RANGE, OVERLAP (destinations; overlapping sources are
  * legal), DUP_ID, NOMEM, CUDA.  nbytes == 0 is legal (no blocks, T = 0).
  * Bytes of a destination beyond nbytes are never written.

@@ -72,6 +72,23 @@ uint64_t blocks_of(uint64_t nbytes) { return nbytes / gms::kBlockBytes + (nbytes
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// The library's own stream for building tables (one per device, made on first use, never destroyed).  It does not
+// synchronise with the default stream, so building a manifest does not wait for whatever else the process has
+// queued on the device -- an engine that is still serving, say.
+cudaError_t build_stream(cudaStream_t *out)
+{
+    static std::mutex mu;
+    static cudaStream_t streams[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!streams[dev] && (e = cudaStreamCreateWithFlags(&streams[dev], cudaStreamNonBlocking)) != cudaSuccess) return e;
+    *out = streams[dev];
+    return cudaSuccess;
+}
+
 // Stable sort of (key, payload) pairs by key.  Validation and list planning sort the tensors' ids, destination and
 // source ranges and short-chunk lengths; with tens of thousands of tensors a comparison sort is then most of the
 // host's build time, so from a few thousand pairs on this is an LSD radix sort, 11 bits at a time, that skips the
@@ -258,8 +275,10 @@ int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vect
             memcpy(h.data(), base.data(), (n + 1) * sizeof(uint64_t));
             if (n) memcpy(h.data() + o_perm, order.data(), n * sizeof(uint32_t));
             uint8_t *tmp = nullptr;
-            e = cudaMalloc(&tmp, bytes);
-            if (e == cudaSuccess) e = cudaMemcpy(tmp, h.data(), bytes, cudaMemcpyHostToDevice);
+            cudaStream_t bs = nullptr;
+            e = build_stream(&bs);
+            if (e == cudaSuccess) e = cudaMalloc(&tmp, bytes);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(tmp, h.data(), bytes, cudaMemcpyHostToDevice, bs);
             ExpandArgs x;
             x.src_offset = m->d_src;
             x.dst = m->d_dst;
@@ -272,8 +291,8 @@ int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vect
             x.n_full = acc;
             x.chunk_blocks = m->chunk_blocks;
             x.out = m->d_by_src;
-            if (e == cudaSuccess) e = launch_expand_chunks(x, nullptr);
-            if (e == cudaSuccess) e = cudaStreamSynchronize(nullptr);
+            if (e == cudaSuccess) e = launch_expand_chunks(x, bs);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(bs);
             if (tmp) cudaFree(tmp);
         } else {
             e = cudaMemcpy(m->d_by_src, sorted.data(), sorted.size() * sizeof(Chunk), cudaMemcpyHostToDevice);
@@ -498,8 +517,10 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             m->d_seg_count = reinterpret_cast<uint32_t *>(m->d_tables + o_segcnt);
             m->d_counter = reinterpret_cast<unsigned int *>(m->d_tables + o_ctr);
             m->d_status = reinterpret_cast<unsigned long long *>(m->d_tables + o_status);
-            e = cudaMemcpy(m->d_tables + o_base, h.data(), h.size(), cudaMemcpyHostToDevice);
-            if (e == cudaSuccess) e = cudaMemset(m->d_tables + o_segcnt, 0, total - o_segcnt);
+            cudaStream_t bs = nullptr;
+            e = build_stream(&bs);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(m->d_tables + o_base, h.data(), h.size(), cudaMemcpyHostToDevice, bs);
+            if (e == cudaSuccess) e = cudaMemsetAsync(m->d_tables + o_segcnt, 0, total - o_segcnt, bs);
             gms::ExpandArgs x;
             x.src_offset = m->d_src = reinterpret_cast<const uint64_t *>(m->d_tables + o_src);
             x.dst = m->d_dst = reinterpret_cast<const uint64_t *>(m->d_tables + o_dst);
@@ -512,14 +533,14 @@ int gms_manifest_build(const gms_entry *entries, size_t n, uint64_t image_bytes,
             x.n_full = plan.n_full;
             x.chunk_blocks = chunk_blocks;
             x.out = m->d_chunks;
-            if (e == cudaSuccess) e = gms::launch_expand_chunks(x, nullptr);
+            if (e == cudaSuccess) e = gms::launch_expand_chunks(x, bs);
             x.full_base = reinterpret_cast<const uint64_t *>(m->d_tables + o_dfb);
             x.tail_pos = reinterpret_cast<const uint32_t *>(m->d_tables + o_dtp);
             x.n_full = dplan.n_full;
             x.chunk_blocks = digest_blocks;
             x.out = m->d_digest_chunks;
-            if (e == cudaSuccess) e = gms::launch_expand_chunks(x, nullptr);
-            if (e == cudaSuccess) e = cudaStreamSynchronize(nullptr);  // the lists are complete when the call returns
+            if (e == cudaSuccess) e = gms::launch_expand_chunks(x, bs);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(bs);  // the lists are complete when the call returns
             if (e == cudaSuccess && env_hook("GMS_CHECK_TABLES", 0, 1, 0)) {
                 // test hook: the device-written lists must equal the host's construction of the same order
                 ensure_host_lists(*m);
