@@ -87,6 +87,40 @@ def test_random_invalid_records_agree_with_oracle(oracle):
     assert agree > 150
 
 
+def test_validation_of_thousands_of_tensors_agrees_with_the_oracle(oracle):
+    """From 2,048 tensors on the library's validation sorts its keys with a radix sort; the oracle's quadratic check
+    of the same records must reach the same verdict -- for a clean record, one duplicated id, one pair of overlapping
+    destinations far apart in the list, and sources that overlap (legal)."""
+    w = W.pack_layout("many", [int(x) for x in np.random.default_rng(5).integers(0, 3000, 5000)], seed=8)
+    base_rows = [(int(r["tensor_id"]), int(r["src_offset"]), int(r["dst_offset"]), int(r["nbytes"])) for r in w.rows]
+    live = [i for i, r in enumerate(base_rows) if r[3] > 64]
+
+    def verdicts(rows):
+        want = oracle.validate(oracle.make_record(rows), w.image_bytes, 1 << 40)
+        ent = gms.make_entries((a, b, FAKE_BASE + c, d) for a, b, c, d in rows)
+        try:
+            m = gms.gms_manifest_build(ent, w.image_bytes, gms.BUILD_HOST_ONLY)
+            n_chunks = gms.gms_manifest_chunk_count(m)
+            covered = sum(gms.gms_manifest_chunk(m, i)[2] for i in range(0, n_chunks, 97))  # the lists still build
+            assert covered > 0
+            m.close()
+            return want, 0
+        except gms.GmsError as e:
+            return want, e.status
+
+    assert verdicts(base_rows) == (oracle.OK, 0)
+    dup = list(base_rows)
+    dup[4321] = (dup[17][0],) + dup[4321][1:]
+    assert verdicts(dup) == (oracle.ERR_DUP_ID, gms.ERR_DUP_ID)
+    ovl = list(base_rows)
+    i, j = live[3], live[-5]
+    ovl[j] = (ovl[j][0], ovl[j][1], ovl[i][2] + 16, ovl[j][3])  # destination j now starts inside destination i
+    assert verdicts(ovl) == (oracle.ERR_OVERLAP, gms.ERR_OVERLAP)
+    shared = list(base_rows)
+    shared[j] = (shared[j][0], shared[i][1], shared[j][2], min(shared[j][3], shared[i][3]))  # same source bytes: legal
+    assert verdicts(shared) == (oracle.OK, 0)
+
+
 def test_index_limits_are_refused_before_anything_is_built():
     # digest slots are 32-bit on the device: 2^32 - 1 blocks or more (16 TiB of payload) is refused during validation
     big = 4096 * (2**32 - 1)
