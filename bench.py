@@ -888,6 +888,41 @@ def e2e_leg(args, torch, gms, bench, dist, dev):
     return out
 
 
+def capture_to_host_leg(torch, gms, bench, reps=3):
+    """gms_capture of the same allocations into a pinned, mapped HOST image (the snapshot direction: device state
+    staged into host memory), against a plain cudaMemcpyAsync device->host of the same bytes into the same buffer."""
+    hptr, dview, arr = gms.gms_host_image_alloc(bench.w.image_bytes)
+    try:
+        cpu = torch.from_numpy(arr)
+        best_copy = None
+        for _ in range(reps + 1):
+            a, b = event_list(torch, 2)
+            a.record()
+            cpu.copy_(bench.image, non_blocking=True)
+            b.record()
+            torch.cuda.synchronize()
+            best_copy = a.elapsed_time(b) if best_copy is None else min(best_copy, a.elapsed_time(b))
+        d2h_gbs = bench.w.image_bytes / best_copy / 1e6
+        times = []
+        for _ in range(reps):
+            a, b = event_list(torch, 2)
+            a.record()
+            gms.gms_capture(bench.m, dview, gms.SRC_HOST_MAPPED, bench.bd, bench.td)
+            b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        gms.gms_verify(bench.m, bench.bd, bench.mm, bench.cap, bench.cnt)
+        ok = bench.check()
+        gbs = bench.payload / min(times) / 1e6
+        return {"call": "gms_capture(host-mapped image): kernel-issued bulk stores across the host link", "ms": min(times),
+                "achieved": gbs, "peak": d2h_gbs, "unit": "GB/s", "frac": gbs / d2h_gbs, "bound": "host_link",
+                "peak_kind": "cudaMemcpyAsync D2H of the image into the same pinned buffer, same run, best of 4",
+                "d2h_bytes": bench.payload, "parity_ok": bool(ok)}
+    finally:
+        torch.cuda.synchronize()
+        gms.gms_host_image_free(hptr)
+
+
 def run_host70b(args, torch, gms, W, dev, index, want_cpu=True, cpu_seconds=4.0):
     """Host-sourced restore of a Llama-3-70B TP8 shard manifest from a pinned, mapped host image,
     against a plain cudaMemcpyAsync of the same bytes from the same allocation.  Returns the config entry."""
@@ -1205,6 +1240,11 @@ def main():
             line["e2e_error"] = str(ex)[:300]
     elif not args.no_e2e:
         line["e2e"] = None
+    if not args.no_e2e and type(bench) is CaptureBench:
+        try:
+            line["capture_to_host"] = capture_to_host_leg(torch, gms, bench)
+        except gms.GmsError as ex:
+            line["capture_to_host"] = {"error": str(ex)[:300]}
 
     if want_cpu and type(bench) in (ManifestBench, CaptureBench):
         fetch = lambda lo, hi: bench.image[lo:hi].cpu().numpy()
