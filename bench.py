@@ -888,6 +888,46 @@ def e2e_leg(args, torch, gms, bench, dist, dev):
     return out
 
 
+def kv_host_legs(torch, gms, bench, reps=3):
+    """The KV subset moved across the host link (Section 6: committed KV blocks kept in host memory): gms_kv_capture of
+    the selected blocks into a pinned, mapped host image and gms_kv_restore back from it, against plain cudaMemcpyAsync
+    of the same number of bytes in each direction through the same pinned buffer."""
+    k = bench.k
+    hptr, dview, arr = gms.gms_host_image_alloc(k.image_bytes)
+    try:
+        cpu = torch.from_numpy(arr)
+        n_sel = len(k.ids)
+
+        def best_of(fn, n):
+            ts = []
+            for _ in range(n):
+                a, b = event_list(torch, 2)
+                a.record()
+                fn()
+                b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            return min(ts)
+
+        d2h = k.image_bytes / best_of(lambda: cpu.copy_(bench.image, non_blocking=True), reps + 1) / 1e6
+        h2d = k.image_bytes / best_of(lambda: bench.image.copy_(cpu, non_blocking=True), reps + 1) / 1e6
+        cap_ms = best_of(lambda: gms.gms_kv_capture(bench.desc, dview, k.img_plane_stride, k.img_slot_stride, gms.SRC_HOST_MAPPED,
+                                                    bench.ids, n_sel, bench.bd_restore, bench.kd, bench.st), reps)
+        ok = bench.st[:2].tolist() == [0, 0]
+        res_ms = best_of(lambda: gms.gms_kv_restore(bench.desc, dview, k.img_plane_stride, k.img_slot_stride, gms.SRC_HOST_MAPPED,
+                                                    bench.ids, n_sel, bench.bd, bench.kd, bench.st), reps)
+        # what was captured from the pool is what is put back: the two calls must report the same digests
+        ok = ok and bench.st[:2].tolist() == [0, 0] and bool(torch.equal(bench.bd, bench.bd_restore))
+        cap, res = bench.payload / cap_ms / 1e6, bench.payload / res_ms / 1e6
+        return {"kv_capture_to_host": {"ms": cap_ms, "achieved": cap, "peak": d2h, "frac": cap / d2h, "unit": "GB/s"},
+                "kv_restore_from_host": {"ms": res_ms, "achieved": res, "peak": h2d, "frac": res / h2d, "unit": "GB/s"},
+                "bound": "host_link", "peak_kind": "cudaMemcpyAsync of the packed image through the same pinned buffer, same run",
+                "bytes": bench.payload, "parity_ok": ok}
+    finally:
+        torch.cuda.synchronize()
+        gms.gms_host_image_free(hptr)
+
+
 def capture_to_host_leg(torch, gms, bench, reps=3):
     """gms_capture of the same allocations into a pinned, mapped HOST image (the snapshot direction: device state
     staged into host memory), against a plain cudaMemcpyAsync device->host of the same bytes into the same buffer."""
@@ -1251,6 +1291,11 @@ def main():
         line["cpu_baseline"] = cpu_baseline_manifest(bench.w, fetch, args.cpu_seconds, all_cores=True)
     elif want_cpu and type(bench) is KvBench:
         line["cpu_baseline"] = cpu_baseline_kv(bench.k, lambda n: bench.image[:n].cpu().numpy())
+    if type(bench) is KvBench and not args.no_e2e:
+        try:
+            line["host_legs"] = kv_host_legs(torch, gms, bench)
+        except gms.GmsError as ex:
+            line["host_legs"] = {"error": str(ex)[:300]}
 
     # ---- all five configurations (single GPU, default invocation only)
     if args.workload is None and world == 1:
@@ -1279,6 +1324,11 @@ def main():
             if name == "tiny":
                 e["note"] = ("latency-bound: 67 MB of traffic is 10 us at the HBM rate; what is measured is launch, "
                              "ramp-up and tail of a 148-CTA persistent kernel")
+            if name == "kv" and not args.no_e2e:
+                try:
+                    e["host_legs"] = kv_host_legs(torch, gms, b)
+                except gms.GmsError as ex:
+                    e["host_legs"] = {"error": str(ex)[:300]}
             if want_cpu and name == "kv":
                 e["cpu_baseline"] = cpu_baseline_kv(b.k, lambda n: b.image[:n].cpu().numpy())
             elif want_cpu:
