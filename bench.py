@@ -1069,6 +1069,8 @@ def run_file(args, torch, gms, W, dev, index, want_cpu=True):
     against (a) the same reader pool filling one pinned buffer with nothing consuming it and (b) the host link."""
     import concurrent.futures as cf
 
+    import numpy as np
+
     bench = ManifestBench("8b", torch, gms, W, dev, fused=False, vmm=args.vmm)
     w = bench.w
     path = os.path.join(args.file_dir, f"gms_bench_image_{os.getpid()}.bin")
@@ -1142,8 +1144,111 @@ def run_file(args, torch, gms, W, dev, index, want_cpu=True):
         if want_cpu:
             fetch = lambda lo, hi: bench.image[lo:hi].cpu().numpy()
             line["cpu_baseline"] = cpu_baseline_manifest(w, fetch, args.cpu_seconds_other, what="manifest (image in host memory)")
-        pipe.close()
         os.close(fd)
+        fd = -1
+        os.remove(path)
+        # ---- the way back: the restored allocations gathered into a new file (gms_capture_fd), against (a) the same
+        # writer threads emptying one pinned buffer into the file with no GPU work and (b) the link, device to host
+        with open(path, "wb") as f:
+            f.truncate(w.image_bytes)
+        wfd = os.open(path, os.O_WRONLY)
+        hptr, _, arr = gms.gms_host_image_alloc(buf_bytes)
+        mv = memoryview(arr)
+
+        def write_all():
+            with cf.ThreadPoolExecutor(n_readers) as ex:
+                for lo in range(0, w.image_bytes, buf_bytes):
+                    n = min(buf_bytes, w.image_bytes - lo)
+                    futs = [ex.submit(os.pwritev, wfd, [mv[o:min(o + slice_b, n)]], lo + o) for o in range(0, n, slice_b)]
+                    for fu in futs:
+                        fu.result()
+
+        write_all()  # the first pass makes the file system allocate the pages
+        t = time.perf_counter()
+        write_all()
+        write_gbs = w.image_bytes / (time.perf_counter() - t) / 1e9
+        cpu_t = torch.from_numpy(arr)
+        ts = []
+        for _ in range(5):
+            e0, e1 = event_list(torch, 2)
+            e0.record()
+            cpu_t.copy_(bench.image[:buf_bytes], non_blocking=True)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        d2h_gbs = buf_bytes / min(ts) / 1e6
+        gms.gms_host_image_free(hptr)
+        bd_capture = torch.zeros_like(bench.bd)
+        gms.gms_capture_fd(bench.m, pipe, wfd, 0, bd_capture, bench.td)
+        cstats = [gms.gms_capture_fd(bench.m, pipe, wfd, 0, bd_capture, bench.td) for _ in range(steps)]
+        os.close(wfd)
+        cbest = min(cstats, key=lambda s: s["total_seconds"])
+        cgbs = w.payload_bytes / cbest["total_seconds"] / 1e9
+
+        def file_ok():
+            """What was written is what was there: a restore fed from the new file must digest to the recorded values."""
+            rfd = os.open(path, os.O_RDONLY)
+            try:
+                bench.bd.zero_()
+                gms.gms_restore_fd(bench.m, pipe, rfd, 0, bench.bd, bench.td)
+            finally:
+                os.close(rfd)
+            gms.gms_verify(bench.m, bench.bd, bench.mm, bench.cap, bench.cnt)
+            return bench.check() and bool(torch.equal(bench.bd, bd_capture))
+
+        cok = file_ok()
+        with open(path, "r+b") as f:  # so that the second pass cannot pass on what the first one wrote
+            for a in range(0, w.image_bytes, 1 << 30):
+                f.seek(a)
+                f.write(bytes(min(1 << 20, w.image_bytes - a)))
+        # the same with the writers storing through a shared mapping of the file (buffered writes to one file are
+        # serialised by the kernel, stores into a mapping are not); yardstick: the same threads copying one pinned
+        # buffer into a mapping of the file
+        import mmap
+
+        wfd = os.open(path, os.O_RDWR)
+        hptr, _, arr = gms.gms_host_image_alloc(buf_bytes)
+
+        def map_all():  # a fresh mapping every pass, as in the call: its pages have to be mapped in again
+            mm = mmap.mmap(wfd, w.image_bytes)
+            mapped = np.frombuffer(mm, dtype=np.uint8)
+
+            def store(lo, o, n):
+                mapped[lo + o:lo + o + n] = arr[o:o + n]
+
+            with cf.ThreadPoolExecutor(n_readers) as ex:
+                for lo in range(0, w.image_bytes, buf_bytes):
+                    n = min(buf_bytes, w.image_bytes - lo)
+                    for fu in [ex.submit(store, lo, o, min(slice_b, n - o)) for o in range(0, n, slice_b)]:
+                        fu.result()
+            del mapped
+            mm.close()
+
+        map_all()
+        t = time.perf_counter()
+        map_all()
+        map_gbs = w.image_bytes / (time.perf_counter() - t) / 1e9
+        gms.gms_host_image_free(hptr)
+        gms.gms_pipe_mapped_writes(pipe, True)
+        gms.gms_capture_fd(bench.m, pipe, wfd, 0, bd_capture, bench.td)
+        mstats = [gms.gms_capture_fd(bench.m, pipe, wfd, 0, bd_capture, bench.td) for _ in range(steps)]
+        gms.gms_pipe_mapped_writes(pipe, False)
+        os.close(wfd)
+        mbest = min(mstats, key=lambda s: s["total_seconds"])
+        mgbs = w.payload_bytes / mbest["total_seconds"] / 1e9
+        mbound = min(map_gbs, d2h_gbs)
+        mok = file_ok() and mbest["mapped_io"] == 1
+        cbound = min(write_gbs, d2h_gbs)
+        line["capture_fd"] = {"value": cgbs, "unit": UNIT, "ms": cbest["total_seconds"] * 1e3, "bound": "storage_write" if write_gbs < d2h_gbs else "host_link",
+                              "peak": cbound, "frac": cgbs / cbound, "writer_yardstick_gbs": write_gbs, "link_yardstick_gbs": d2h_gbs,
+                              "peak_kind": "min(same writer threads and slicing emptying one pinned buffer into the same file with no producer; "
+                                           "plain cudaMemcpyAsync D2H of one pinned buffer)", "pipe_stats_best": cbest, "parity_ok": bool(cok)}
+        line["capture_fd_mapped"] = {"value": mgbs, "unit": UNIT, "ms": mbest["total_seconds"] * 1e3, "bound": "storage_write" if map_gbs < d2h_gbs else "host_link",
+                                     "peak": mbound, "frac": mgbs / mbound, "writer_yardstick_gbs": map_gbs, "link_yardstick_gbs": d2h_gbs,
+                                     "peak_kind": "min(same threads and slicing copying one pinned buffer into a shared mapping of the same file; "
+                                                  "plain cudaMemcpyAsync D2H of one pinned buffer)", "pipe_stats_best": mbest,
+                                     "parity_ok": bool(mok)}
+        pipe.close()
         bench.close()
         return line
     finally:

@@ -404,11 +404,38 @@ typedef struct {
     double total_seconds;      /* wall time of the call                                     */
     uint32_t direct_io;        /* 1: the file system accepted O_DIRECT reads                */
     uint32_t copy_engine;      /* 1: windows went pinned buffer -> copy engine -> device    */
+    uint32_t mapped_io;        /* 1: gms_capture_fd stored through a mapping of the file    */
+    uint32_t reserved;
 } gms_pipe_stats;
 int gms_pipe_create(uint32_t n_buffers, uint64_t buffer_bytes, uint32_t n_readers, gms_pipe **out);
 int gms_pipe_direct_io(gms_pipe *p, int enable);
+int gms_pipe_mapped_writes(gms_pipe *p, int enable);
 int gms_pipe_destroy(gms_pipe *p);
 int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_offset, uint64_t *d_block_digests,
+                   uint64_t *d_tensor_digests, void *stream, gms_pipe_stats *stats);
+
+/*
+ * gms_capture_fd -- the way back through the same pipe: Section 3.1, steps 3 and 4 (device state is staged
+ * into host memory and serialised to durable storage).  gms_capture, window by window: the kernel gathers
+ * each window of the image straight into one of the pipe's pinned buffers (kernel-issued stores cross the
+ * link at the copy engine's rate in this direction, so the device buffers are not used) and the pipe's
+ * threads write it out with pwrite() while the next window is gathered.  File byte file_offset + k = image
+ * byte k for every byte a tensor covers; bytes of the file between tensors' ranges are not written, and the
+ * file is neither truncated nor synced (the caller's fsync decides when it is durable).  Digests as from
+ * gms_capture.  `fd` must be open for writing; gms_pipe_direct_io does not apply.  Synchronous like
+ * gms_restore_fd; in `stats`, bytes_read counts the bytes written and wait_read_seconds the time spent
+ * waiting for the writers.  Errors: NULL, ARG, OVERLAP (tensors share image bytes), NOMEM, STATE, IO
+ * (write error), CUDA.
+ * gms_pipe_mapped_writes(p, 1): the writers store through a shared mapping of the file instead of calling
+ * pwrite().  The kernel lets only one buffered write at a time into a file, so pwrite from many threads
+ * runs at one core's copy rate; stores into a mapping run on all of them.  Meant for snapshots kept in
+ * the page cache or on tmpfs.  Used only when `fd` is a regular file, open for reading and writing, that
+ * already spans file_offset + the image (it is never extended), else pwrite is used as before
+ * (stats.mapped_io says which).  The caller must have the file's blocks in that range allocated
+ * (written before, or posix_fallocate): a store into a hole of a full file system raises SIGBUS, where
+ * pwrite would have returned an error.  Off unless asked for.
+ */
+int gms_capture_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_offset, uint64_t *d_block_digests,
                    uint64_t *d_tensor_digests, void *stream, gms_pipe_stats *stats);
 
 /*

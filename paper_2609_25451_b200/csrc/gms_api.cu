@@ -349,8 +349,18 @@ int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vect
     return GMS_OK;
 }
 
+int manifest_sorted_sources(const gms_manifest *m, std::vector<std::pair<uint64_t, uint64_t>> *out)
+{
+    if (!m->sources_disjoint) return GMS_ERR_OVERLAP;
+    out->clear();
+    for (const gms_entry &e : m->entries)
+        if (e.nbytes) out->emplace_back(e.src_offset, e.nbytes);
+    std::sort(out->begin(), out->end());
+    return GMS_OK;
+}
+
 int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void *window_base, bool first,
-                           uint64_t *d_block_digests, uint64_t *d_tensor_digests, cudaStream_t s)
+                           uint64_t *d_block_digests, uint64_t *d_tensor_digests, cudaStream_t s, bool capture)
 {
     StreamArgs a;
     a.chunks = m->d_by_src + w.first_chunk;
@@ -363,7 +373,7 @@ int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void
     a.status = m->d_status;
     a.n_counters = 1;
     a.group = 1;
-    a.capture = 0;
+    a.capture = capture ? 1u : 0u;
     a.keep_accum = first ? 0u : 1u;
     a.stall_chunk = 0xffffffffu;
     a.expected = nullptr;

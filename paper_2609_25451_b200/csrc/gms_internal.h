@@ -5,6 +5,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstdlib>
+#include <utility>
 #include <vector>
 
 #include <cuda_runtime.h>
@@ -140,7 +141,11 @@ namespace gms {
 // a device copy of the chunk list sorted by source offset).  Returns a GMS_* status.
 int manifest_src_windows(const gms_manifest *m, uint64_t buffer_bytes, std::vector<SrcWindow> *out);
 // Enqueues the restore of one window; `window_base` is the device-accessible address of image byte w.src_lo.
+// With `capture` the window is written instead (allocations -> window), by the same kernel.
 int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void *window_base, bool first,
-                           uint64_t *d_block_digests, uint64_t *d_tensor_digests, cudaStream_t s);
+                           uint64_t *d_block_digests, uint64_t *d_tensor_digests, cudaStream_t s, bool capture = false);
+// The image ranges (offset, length) of the non-empty tensors in ascending order of offset; GMS_ERR_OVERLAP if two
+// tensors share image bytes.
+int manifest_sorted_sources(const gms_manifest *m, std::vector<std::pair<uint64_t, uint64_t>> *out);
 uint64_t manifest_n_tensors(const gms_manifest *m);
 }  // namespace gms

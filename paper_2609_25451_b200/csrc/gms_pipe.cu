@@ -1,4 +1,4 @@
-// gms_restore_fd: storage -> pinned host buffers -> device allocations, pipelined.
+// gms_restore_fd: storage -> pinned host buffers -> device allocations, pipelined; gms_capture_fd: the way back.
 //
 // Section 4 (GMS paragraph) has a fresh writer fill a cold service from storage while the process
 // itself is being restored; Section 3.1 prices that at S / B_eff and Section 3.3 notes that restoring
@@ -12,17 +12,22 @@
 // the kernel that read it has (CUDA events).  If the device buffers cannot be had, the kernel reads the
 // pinned buffers across the host link instead (about 7 % slower on the link).
 // All waiting is on the host (condition variables, cudaEventSynchronize); no kernel waits for a flag.
+#include <algorithm>
 #include <condition_variable>
 #include <cerrno>
+#include <cstring>
 #include <chrono>
 #include <deque>
 #include <functional>
 #include <mutex>
 #include <thread>
+#include <utility>
 #include <vector>
 
 #include <atomic>
 #include <fcntl.h>
+#include <sys/mman.h>
+#include <sys/stat.h>
 #include <unistd.h>
 
 #include "../../include/gms.h"
@@ -105,6 +110,7 @@ struct gms_pipe {
     cudaStream_t copy_stream = nullptr;
     uint64_t dev_uses = 0;              // windows pushed through the device ring so far (across calls)
     bool direct_io = false;             // gms_pipe_direct_io: read with O_DIRECT where the file system allows it
+    bool mapped_writes = false;         // gms_pipe_mapped_writes: gms_capture_fd stores through a shared mapping of the file
     ReaderPool *pool = nullptr;
     std::mutex busy;             // one restore at a time per pipe
 };
@@ -281,6 +287,14 @@ int gms_pipe_direct_io(gms_pipe *p, int enable)
     if (!p) return GMS_ERR_NULL;
     std::lock_guard<std::mutex> one(p->busy);
     p->direct_io = enable != 0;
+    return GMS_OK;
+}
+
+int gms_pipe_mapped_writes(gms_pipe *p, int enable)
+{
+    if (!p) return GMS_ERR_NULL;
+    std::lock_guard<std::mutex> one(p->busy);
+    p->mapped_writes = enable != 0;
     return GMS_OK;
 }
 
@@ -468,6 +482,165 @@ int gms_restore_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_off
     if (e != cudaSuccess && rc == GMS_OK) rc = gms::report_cuda_error(e);
     st.direct_io = dfd >= 0 && direct_ok.load() ? 1u : 0u;
     st.copy_engine = staged ? 1u : 0u;
+    st.total_seconds = now_s() - t_start;
+    if (stats) *stats = st;
+    if (io_error) return GMS_ERR_IO;
+    return rc;
+}
+
+// The other direction: device allocations -> pinned buffers -> file (Section 3.1: step 3 stages device state into
+// host memory, step 4 serialises it to durable storage).  The capture kernel gathers one window of the image at a
+// time straight into a pinned buffer (kernel-issued bulk stores across the host link run at the rate of the copy
+// engine in this direction, so there is no device-side staging), and the pipe's threads write the window's tensor
+// ranges to the file with pwrite while the kernel fills the next buffer.  Only bytes that belong to a tensor are
+// written: what the file holds between two tensors' ranges stays as it was.
+int gms_capture_fd(const gms_manifest *m, gms_pipe *p, int fd, uint64_t file_offset, uint64_t *d_block_digests,
+                   uint64_t *d_tensor_digests, void *stream, gms_pipe_stats *stats)
+{
+    if (!m || !p) return GMS_ERR_NULL;
+    if (fd < 0) return GMS_ERR_ARG;
+    std::lock_guard<std::mutex> one(p->busy);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<std::pair<uint64_t, uint64_t>> ranges;  // image ranges of the tensors, ascending
+    int rc = gms::manifest_sorted_sources(m, &ranges);
+    if (rc != GMS_OK) return rc;
+    std::vector<gms::SrcWindow> windows;
+    rc = gms::manifest_src_windows(m, p->buffer_bytes, &windows);
+    if (rc != GMS_OK) return rc;
+    const double t_start = now_s();
+    gms_pipe_stats st = {};
+    st.windows = windows.size();
+    if (windows.empty()) {  // nothing to move: still clear the accumulators
+        gms::SrcWindow none = {0, 0, 0, 0};
+        rc = gms::manifest_launch_window(m, none, p->dview[0], true, d_block_digests, d_tensor_digests, s, true);
+    }
+
+    // On request (gms_pipe_mapped_writes): the writers copy into a shared mapping of the file instead of calling pwrite.
+    // Buffered writes to one file are serialised by the kernel (one writer holds the file's lock at a time), stores
+    // into a mapping are not, so for a file that lives in the page cache this is the difference between one core's
+    // copy rate and all of them.  Only for a regular file that already spans the image (a store beyond the end of
+    // the file would raise SIGBUS) on a descriptor that allows a shared writable mapping; pwrite otherwise.
+    uint8_t *map = nullptr;
+    uint64_t map_lo = 0, map_len = 0;
+    if (p->mapped_writes && !windows.empty()) {
+        struct stat sb;
+        const uint64_t lo = file_offset + windows.front().src_lo, hi = file_offset + windows.back().src_hi;
+        if (fstat(fd, &sb) == 0 && S_ISREG(sb.st_mode) && (uint64_t)sb.st_size >= hi) {
+            map_lo = lo & ~(uint64_t)4095;
+            map_len = hi - map_lo;
+            void *a = mmap(nullptr, map_len, PROT_READ | PROT_WRITE, MAP_SHARED, fd, (off_t)map_lo);
+            if (a != MAP_FAILED) map = static_cast<uint8_t *>(a);
+        }
+    }
+    st.mapped_io = map ? 1u : 0u;
+
+    struct Piece {
+        uint64_t buf_off, file_off, n;
+    };
+    std::vector<WindowReads> writes(windows.size());  // completion state of each window's writes
+    const uint32_t n_writers = p->pool->size();
+    size_t next_launch = 0, next_write = 0, ri = 0;  // ri: first tensor range that reaches into the window to write
+    int io_error = 0;
+    auto wait_written = [&](size_t w) {
+        const double t0 = now_s();
+        std::unique_lock<std::mutex> l(writes[w].mu);
+        writes[w].cv.wait(l, [&] { return writes[w].pending == 0; });
+        st.wait_read_seconds += now_s() - t0;
+        if (writes[w].error && !io_error) io_error = writes[w].error;
+    };
+    while (rc == GMS_OK && !io_error && next_write < windows.size()) {
+        // gather as far ahead as the ring allows: a buffer is free once the window it held has been written out
+        while (next_launch < windows.size() && next_launch < next_write + p->n_buffers) {
+            if (next_launch >= p->n_buffers) wait_written(next_launch - p->n_buffers);
+            if (io_error) break;
+            const uint32_t b = (uint32_t)(next_launch % p->n_buffers);
+            rc = gms::manifest_launch_window(m, windows[next_launch], p->dview[b], next_launch == 0, d_block_digests,
+                                             d_tensor_digests, s, true);
+            if (rc != GMS_OK) break;
+            cudaError_t e = cudaEventRecord(p->done[b], s);
+            if (e != cudaSuccess) {
+                rc = gms::report_cuda_error(e);
+                break;
+            }
+            ++next_launch;
+        }
+        if (rc != GMS_OK || io_error) break;
+        // the window to write next: wait for its kernel, then hand its tensor ranges to the writers
+        const gms::SrcWindow &w = windows[next_write];
+        const uint32_t b = (uint32_t)(next_write % p->n_buffers);
+        {
+            const double t0 = now_s();
+            cudaError_t e = cudaEventSynchronize(p->done[b]);
+            st.wait_gpu_seconds += now_s() - t0;
+            if (e != cudaSuccess) {
+                rc = gms::report_cuda_error(e);
+                break;
+            }
+        }
+        // the tensor bytes inside [src_lo, src_hi), adjacent ranges merged, cut into jobs of about a writer's share
+        uint64_t slice = (w.src_hi - w.src_lo + n_writers - 1) / n_writers;
+        slice = std::max<uint64_t>((slice + (1u << 20) - 1) & ~((uint64_t)(1u << 20) - 1), 1u << 20);
+        std::vector<std::vector<Piece>> jobs(1);
+        uint64_t job_bytes = 0;
+        while (ri < ranges.size() && ranges[ri].first + ranges[ri].second <= w.src_lo) ++ri;
+        for (size_t k = ri; k < ranges.size() && ranges[k].first < w.src_hi; ++k) {
+            uint64_t lo = std::max(ranges[k].first, w.src_lo);
+            const uint64_t hi = std::min(ranges[k].first + ranges[k].second, w.src_hi);
+            while (lo < hi) {
+                const uint64_t n = std::min(hi - lo, slice - job_bytes);
+                std::vector<Piece> &job = jobs.back();
+                if (!job.empty() && job.back().buf_off + job.back().n == lo - w.src_lo)
+                    job.back().n += n;  // continues the piece before it
+                else
+                    job.push_back({lo - w.src_lo, file_offset + lo, n});
+                lo += n;
+                job_bytes += n;
+                st.bytes_read += n;
+                if (job_bytes == slice) jobs.emplace_back(), job_bytes = 0;
+            }
+        }
+        if (jobs.back().empty()) jobs.pop_back();
+        WindowReads &wr = writes[next_write];
+        wr.pending = (uint32_t)jobs.size();
+        const uint8_t *base = static_cast<const uint8_t *>(p->host[b]);
+        for (std::vector<Piece> &job : jobs)
+            p->pool->submit([fd, base, map, map_lo, &wr, pieces = std::move(job)] {
+                int err = 0;
+                for (const Piece &pc : pieces) {
+                    if (map) {
+                        uint8_t *to = map + (pc.file_off - map_lo);
+#ifdef MADV_POPULATE_WRITE
+                        // map the piece's pages in one call instead of one fault per page (a hint: errors do not matter)
+                        if (pc.n >= (1u << 16)) {
+                            uint8_t *lo = reinterpret_cast<uint8_t *>(reinterpret_cast<uint64_t>(to) & ~(uint64_t)4095);
+                            (void)madvise(lo, (size_t)(to + pc.n - lo), MADV_POPULATE_WRITE);
+                        }
+#endif
+                        memcpy(to, base + pc.buf_off, pc.n);
+                        continue;
+                    }
+                    uint64_t put = 0;
+                    while (put < pc.n && !err) {
+                        const ssize_t r = pwrite(fd, base + pc.buf_off + put, pc.n - put, (off_t)(pc.file_off + put));
+                        if (r < 0 && errno == EINTR) continue;
+                        if (r <= 0)
+                            err = (r < 0 && errno) ? errno : -1;
+                        else
+                            put += (uint64_t)r;
+                    }
+                    if (err) break;
+                }
+                std::lock_guard<std::mutex> l(wr.mu);
+                if (err && !wr.error) wr.error = err;
+                if (--wr.pending == 0) wr.cv.notify_all();
+            });
+        ++next_write;
+    }
+    // drain: writers use the pipe's buffers and `writes`, kernels write the buffers: neither may outlive this call
+    for (size_t w = 0; w < next_write; ++w) wait_written(w);
+    if (map) munmap(map, map_len);
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess && rc == GMS_OK) rc = gms::report_cuda_error(e);
     st.total_seconds = now_s() - t_start;
     if (stats) *stats = st;
     if (io_error) return GMS_ERR_IO;

@@ -35,7 +35,7 @@ EXPORTS = (
     "gms_manifest_build", "gms_manifest_destroy", "gms_manifest_info", "gms_manifest_block_base",
     "gms_manifest_chunk_count", "gms_manifest_chunk", "gms_manifest_set_expected", "gms_restore", "gms_capture", "gms_digest",
     "gms_verify", "gms_digest_verify", "gms_restore_verify", "gms_verify_tensors", "gms_verify_flat_noalloc", "gms_last_device_status", "gms_kv_restore", "gms_kv_capture", "gms_kv_digest", "gms_kv_verify", "gms_host_image_alloc", "gms_host_image_free",
-    "gms_pipe_create", "gms_pipe_direct_io", "gms_pipe_destroy", "gms_restore_fd", "gms_stage_create", "gms_stage_destroy", "gms_restore_staged",
+    "gms_pipe_create", "gms_pipe_direct_io", "gms_pipe_mapped_writes", "gms_pipe_destroy", "gms_restore_fd", "gms_capture_fd", "gms_stage_create", "gms_stage_destroy", "gms_restore_staged",
     "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
     "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
     "gms_service_detach", "gms_service_reattach", "gms_service_release_pages", "gms_service_back_pages",
@@ -98,8 +98,10 @@ def lib():
             "gms_host_image_free": (i, [p]),
             "gms_pipe_create": (i, [u32, u64, u32, pp]),
             "gms_pipe_direct_io": (i, [p, i]),
+            "gms_pipe_mapped_writes": (i, [p, i]),
             "gms_pipe_destroy": (i, [p]),
             "gms_restore_fd": (i, [p, p, i, u64, p, p, p, p]),
+            "gms_capture_fd": (i, [p, p, i, u64, p, p, p, p]),
             "gms_stage_create": (i, [u32, u64, pp]),
             "gms_stage_destroy": (i, [p]),
             "gms_restore_staged": (i, [p, p, p, p, p, p]),
@@ -301,7 +303,7 @@ def gms_host_image_free(host_ptr: int):
 class PipeStats(C.Structure):
     _fields_ = [("windows", C.c_uint64), ("bytes_read", C.c_uint64), ("wait_read_seconds", C.c_double),
                 ("wait_gpu_seconds", C.c_double), ("total_seconds", C.c_double), ("direct_io", C.c_uint32),
-                ("copy_engine", C.c_uint32)]
+                ("copy_engine", C.c_uint32), ("mapped_io", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class Pipe:
@@ -328,11 +330,23 @@ def gms_pipe_direct_io(pipe: Pipe, enable: bool):
     _check(lib().gms_pipe_direct_io(pipe.handle, 1 if enable else 0), "gms_pipe_direct_io")
 
 
+def gms_pipe_mapped_writes(pipe: Pipe, enable: bool):
+    _check(lib().gms_pipe_mapped_writes(pipe.handle, 1 if enable else 0), "gms_pipe_mapped_writes")
+
+
 def gms_restore_fd(m: Manifest, pipe: Pipe, fd: int, file_offset: int, d_block_digests, d_tensor_digests, stream=None) -> dict:
     """Synchronous; returns the call's statistics as a dict."""
     st = PipeStats()
     _check(lib().gms_restore_fd(m.handle, pipe.handle, int(fd), int(file_offset), _dev(d_block_digests),
                                 _dev(d_tensor_digests), _stream(stream), C.byref(st)), "gms_restore_fd")
+    return {k: getattr(st, k) for k, _ in PipeStats._fields_}
+
+
+def gms_capture_fd(m: Manifest, pipe: Pipe, fd: int, file_offset: int, d_block_digests, d_tensor_digests, stream=None) -> dict:
+    """Synchronous; returns the call's statistics as a dict (``bytes_read`` counts the bytes written)."""
+    st = PipeStats()
+    _check(lib().gms_capture_fd(m.handle, pipe.handle, int(fd), int(file_offset), _dev(d_block_digests),
+                                _dev(d_tensor_digests), _stream(stream), C.byref(st)), "gms_capture_fd")
     return {k: getattr(st, k) for k, _ in PipeStats._fields_}
 
 

@@ -28,7 +28,7 @@ int main(void)
         (fn)gms_manifest_chunk_count, (fn)gms_manifest_chunk, (fn)gms_manifest_set_expected, (fn)gms_restore,
         (fn)gms_capture, (fn)gms_digest, (fn)gms_verify, (fn)gms_digest_verify, (fn)gms_restore_verify, (fn)gms_verify_tensors, (fn)gms_verify_flat_noalloc,
         (fn)gms_last_device_status, (fn)gms_kv_restore, (fn)gms_kv_capture, (fn)gms_kv_digest, (fn)gms_kv_verify, (fn)gms_host_image_alloc,
-        (fn)gms_host_image_free, (fn)gms_pipe_create, (fn)gms_pipe_direct_io, (fn)gms_pipe_destroy, (fn)gms_restore_fd, (fn)gms_stage_create,
+        (fn)gms_host_image_free, (fn)gms_pipe_create, (fn)gms_pipe_direct_io, (fn)gms_pipe_mapped_writes, (fn)gms_pipe_destroy, (fn)gms_restore_fd, (fn)gms_capture_fd, (fn)gms_stage_create,
         (fn)gms_stage_destroy, (fn)gms_restore_staged, (fn)gms_service_create, (fn)gms_service_destroy,
         (fn)gms_service_acquire_rw, (fn)gms_service_alloc, (fn)gms_service_commit, (fn)gms_service_abort,
         (fn)gms_service_acquire_ro, (fn)gms_service_release_ro, (fn)gms_service_info, (fn)gms_service_access,

@@ -3,7 +3,8 @@ result must be exactly what gms_restore produces from the same bytes, so the ora
 file's contents is the reference: destination bytes, block digests, tensor digests, bit-exact -- with
 buffers far smaller than the tensors (tensors span many windows), file offsets that are 4 KiB-aligned
 (windows read with O_DIRECT where the file system takes it), 16-byte-aligned and odd, odd sizes, and
-the error paths (short file, bad arguments)."""
+the error paths (short file, bad arguments).  gms_capture_fd, the way back, must leave in the file exactly what the
+oracle's capture leaves in an image: every tensor's bytes in place, every byte between them as it was."""
 import ctypes
 import os
 
@@ -28,7 +29,9 @@ def test_pipe_argument_checks_need_no_gpu():
     assert L.gms_pipe_create(2, 1 << 20, 4, None) == gms.ERR_NULL
     assert L.gms_pipe_destroy(None) == gms.OK
     assert L.gms_pipe_direct_io(None, 1) == gms.ERR_NULL
+    assert L.gms_pipe_mapped_writes(None, 1) == gms.ERR_NULL
     assert L.gms_restore_fd(None, None, 0, 0, None, None, None, None) == gms.ERR_NULL
+    assert L.gms_capture_fd(None, None, 0, 0, None, None, None, None) == gms.ERR_NULL
     assert "file" in gms.gms_strerror(gms.ERR_IO)
 
 
@@ -205,3 +208,142 @@ def test_restore_fd_empty_manifest(tmp_path):
         os.close(fd)
         pipe.close()
         d.close()
+
+
+PATTERN = 0xA5  # what the file holds before a capture
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("n_buffers,buffer_mib,n_writers,file_offset",
+                         [(2, 1, 1, 0), (3, 2, 4, 4096 + 16), (4, 16, 8, 5), (2, 4, 3, 8192)])
+def test_capture_fd_leaves_in_the_file_what_the_oracle_captures(oracle, tmp_path, n_buffers, buffer_mib, n_writers, file_offset):
+    from gpu_harness import payload_of
+
+    w = W.mixed_manifest(n_small=1500, n_large=3, large_bytes=(7 << 20) + 40, round16=False, seed=124)
+    tail = 100  # bytes of the file behind the image: must stay untouched as well
+    path = str(tmp_path / "snapshot.bin")
+    d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    pipe = gms.gms_pipe_create(n_buffers, buffer_mib << 20, n_writers)
+    try:
+        for seed in (31, 32):  # twice with different contents: nothing of the first pass may show in the second file
+            slab_h = W.random_bytes_host(w.slab_bytes, seed=seed)
+            d.slab.copy_(torch.from_numpy(slab_h))
+            want = np.full(w.image_bytes, PATTERN, np.uint8)
+            rc, obd, otd = oracle.capture(oracle_record(oracle, w), want, slab_h)
+            assert rc == 0
+            with open(path, "wb") as f:
+                f.write(bytes([PATTERN]) * (file_offset + w.image_bytes + tail))
+            # second pass: the writers store through a shared mapping of the file (needs a descriptor that may be mapped)
+            mapped = seed == 32
+            gms.gms_pipe_mapped_writes(pipe, mapped)
+            fd = os.open(path, os.O_RDWR if mapped else os.O_WRONLY)
+            try:
+                d.reset_outputs()
+                st = gms.gms_capture_fd(d.m, pipe, fd, file_offset, d.bd_ptr(), d.td_ptr())
+            finally:
+                os.close(fd)
+            assert gms.gms_last_device_status(d.m) == 0 and st["mapped_io"] == (1 if mapped else 0)
+            got = np.fromfile(path, dtype=np.uint8)
+            assert got.size == file_offset + w.image_bytes + tail, "the file's length changed"
+            assert (got[:file_offset] == PATTERN).all() and (got[file_offset + w.image_bytes:] == PATTERN).all()
+            assert np.array_equal(got[file_offset:file_offset + w.image_bytes], want), "tensor bytes or the gaps between them differ"
+            assert np.array_equal(payload_of(d.bd, d.nb), obd) and np.array_equal(payload_of(d.td, d.nt), otd)
+            assert np.array_equal(d.slab_host(), slab_h), "capture wrote to the allocations"
+            assert st["bytes_read"] == sum(int(r["nbytes"]) for r in w.rows)
+            assert st["windows"] >= w.image_bytes // (buffer_mib << 20)
+        # and back: a restore fed from that file reproduces the allocations it was captured from
+        d.slab.fill_(FILL)
+        fd = os.open(path, os.O_RDONLY)
+        try:
+            d.reset_outputs()
+            gms.gms_restore_fd(d.m, pipe, fd, file_offset, d.bd_ptr(), d.td_ptr())
+        finally:
+            os.close(fd)
+        assert np.array_equal(payload_of(d.bd, d.nb), obd) and np.array_equal(payload_of(d.td, d.nt), otd)
+        back = d.slab_host()
+        for r in w.rows:
+            o, n = int(r["dst_offset"]), int(r["nbytes"])
+            assert np.array_equal(back[o:o + n], slab_h[o:o + n])
+    finally:
+        pipe.close()
+        d.close()
+
+
+@pytest.mark.gpu
+def test_capture_fd_error_paths(tmp_path):
+    w = W.pack_layout("cap-err", [3 << 20, 0, 100], seed=6)
+    d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    d.slab.copy_(torch.from_numpy(W.random_bytes_host(w.slab_bytes, seed=9)))
+    pipe = gms.gms_pipe_create(2, 1 << 20, 2)
+    path = str(tmp_path / "ro.bin")
+    with open(path, "wb") as f:
+        f.write(b"\0" * w.image_bytes)
+    fd = os.open(path, os.O_RDONLY)  # not open for writing: every pwrite fails
+    try:
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_capture_fd(d.m, pipe, fd, 0, None, None)
+        assert ei.value.status == gms.ERR_IO
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_capture_fd(d.m, pipe, -1, 0, None, None)
+        assert ei.value.status == gms.ERR_ARG
+    finally:
+        os.close(fd)
+    # the pipe and the manifest remain usable after the error; mapped writes were asked for but this descriptor cannot be
+    # mapped for writing (write-only), so pwrite is used
+    gms.gms_pipe_mapped_writes(pipe, True)
+    fd = os.open(path, os.O_WRONLY)
+    try:
+        st = gms.gms_capture_fd(d.m, pipe, fd, 0, None, None)
+        assert st["mapped_io"] == 0
+    finally:
+        os.close(fd)
+    # nor is a file that ends before the image does ever mapped (or extended by the mapping): pwrite grows it
+    short = str(tmp_path / "short.bin")
+    with open(short, "wb") as f:
+        f.write(b"\0" * 4096)
+    fd = os.open(short, os.O_RDWR)
+    try:
+        st = gms.gms_capture_fd(d.m, pipe, fd, 0, None, None)
+        assert st["mapped_io"] == 0
+    finally:
+        os.close(fd)
+    for written in (path, short):
+        got = np.fromfile(written, dtype=np.uint8)
+        for r in w.rows:
+            s, o, n = int(r["src_offset"]), int(r["dst_offset"]), int(r["nbytes"])
+            assert np.array_equal(got[s:s + n], d.slab[o:o + n].cpu().numpy())
+    # tensors that share image bytes cannot be captured
+    base = d.slab.data_ptr()
+    shared = gms.make_entries([(1, 0, base, 4096), (2, 0, base + 8192, 4096)])
+    m2 = gms.gms_manifest_build(shared, 4096)
+    fd = os.open(path, os.O_WRONLY)
+    try:
+        with pytest.raises(gms.GmsError) as ei:
+            gms.gms_capture_fd(m2, pipe, fd, 0, None, None)
+        assert ei.value.status == gms.ERR_OVERLAP
+    finally:
+        os.close(fd)
+        m2.close()
+        pipe.close()
+        d.close()
+
+
+@pytest.mark.gpu
+def test_capture_fd_empty_manifest(tmp_path):
+    from gpu_harness import payload_of
+
+    w = W.pack_layout("empty", [0, 0], seed=1)
+    path = str(tmp_path / "e.bin")
+    _write_image(path, np.full(16, PATTERN, np.uint8), 0)
+    d = DeviceWorkload(w, image_dev=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    pipe = gms.gms_pipe_create(2, 1 << 20, 1)
+    fd = os.open(path, os.O_WRONLY)
+    try:
+        d.reset_outputs()
+        st = gms.gms_capture_fd(d.m, pipe, fd, 0, d.bd_ptr(), d.td_ptr())
+        assert st["windows"] == 0 and st["bytes_read"] == 0 and (payload_of(d.td, d.nt) == 0).all()
+    finally:
+        os.close(fd)
+        pipe.close()
+        d.close()
+    assert (np.fromfile(path, dtype=np.uint8) == PATTERN).all()
