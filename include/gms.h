@@ -464,8 +464,9 @@ int gms_restore_staged(const gms_manifest *m, gms_stage *st, const void *host_im
  * slabs for larger allocations, permissions set per slab) and Section 3.2 (ownership protocol:
  * EMPTY -> RW, one writer populates -> COMMITTED, immutable -> RO while n >= 1 readers hold it;
  * a writer that gives up before commit discards everything; write access returns after the last
- * reader has left; read-only is enforced with cuMemSetAccess).  One process, current device; the
- * separate service process and descriptor passing of the paper are not part of this library.
+ * reader has left; read-only is enforced with cuMemSetAccess).  Current device.  The state machine
+ * lives in the process that created the service; other processes take part through the export / import
+ * calls further down.
  *   create      slab_bytes = 0 means 2 GiB; GMS_SERVICE_DRY_RUN keeps the books without any CUDA
  *               call (addresses are made up and must not be dereferenced)
  *   acquire_rw  EMPTY -> RW, or COMMITTED -> RW (contents and addresses kept, slabs writable again);
@@ -486,6 +487,7 @@ int gms_restore_staged(const gms_manifest *m, gms_stage *st, const void *host_im
 #define GMS_STATE_COMMITTED 2u
 #define GMS_STATE_RO 3u
 #define GMS_SERVICE_DRY_RUN 1u
+#define GMS_SERVICE_SHAREABLE 2u /* slabs can be handed to other processes (gms_service_export_fd) */
 typedef struct gms_service gms_service; /* opaque */
 typedef struct {
     uint32_t state, readers;
@@ -529,6 +531,44 @@ int gms_service_detach(gms_service *s);
 int gms_service_reattach(gms_service *s);
 int gms_service_release_pages(gms_service *s);
 int gms_service_back_pages(gms_service *s);
+
+/*
+ * Across processes -- Section 4, GMS paragraph (the service process creates the physical allocations and
+ * keeps their handles; clients receive them as file descriptors over Unix sockets, import them, map them and
+ * set their own access) and Section 3.2 (the memory therefore outlives the engine process that filled or used
+ * it, and the replacement engine attaches it read-only).  The library provides the two ends; the socket and
+ * whatever is said on it (who holds the service in which state) belong to the processes that use them.
+ *   gms_service_slab       size and address of slab `index` (0 .. n_slabs-1 of gms_service_info) in the service's
+ *                          own address space, so that allocation addresses can be written as (slab, offset)
+ *   gms_service_export_fd  a new file descriptor for slab `index` (service created with GMS_SERVICE_SHAREABLE;
+ *                          GMS_ERR_STATE otherwise, in a dry run, or without pages); the caller sends it with
+ *                          SCM_RIGHTS and closes its copy.  The memory lives as long as any process holds a
+ *                          handle or a mapping of it.
+ *   gms_import_create      the client's side, on the same GPU (the current device): imports the n descriptors
+ *                          (which stay open; the caller closes them), reserves address space for each -- at
+ *                          slabs[i].address where that is free -- maps it and sets this process's access:
+ *                          read-only, or writable with GMS_IMPORT_WRITABLE (the writer that populates, RW in the
+ *                          protocol).  GMS_IMPORT_SAME_ADDRESS: fail with GMS_ERR_RANGE unless every slab lands
+ *                          at the service's address (an engine restored from a snapshot has those addresses in its
+ *                          graphs and metadata, and kept the ranges free; a fresh process will often find them
+ *                          taken); without it any address will do and gms_import_address tells which.  Permissions are per process: a reader's mapping stays read-only whatever the
+ *                          others hold.
+ *   gms_import_destroy     synchronises the device, unmaps, frees the address ranges and drops the handles; the
+ *                          contents stay with the service.
+ * Errors: NULL, ARG, RANGE, STATE, NOMEM, CUDA.
+ */
+#define GMS_IMPORT_WRITABLE 1u
+#define GMS_IMPORT_SAME_ADDRESS 2u
+typedef struct {
+    uint64_t address, bytes;
+    uint32_t dedicated, reserved;
+} gms_slab_info;
+typedef struct gms_import gms_import; /* opaque */
+int gms_service_slab(gms_service *s, uint64_t index, gms_slab_info *out);
+int gms_service_export_fd(gms_service *s, uint64_t index, int *fd);
+int gms_import_create(const int *fds, const gms_slab_info *slabs, size_t n, uint32_t flags, gms_import **out);
+int gms_import_address(const gms_import *imp, size_t index, void **dptr);
+int gms_import_destroy(gms_import *imp);
 
 /*
  * Tuning and test hooks.  The library reads the environment variables below once per process (the chunk lengths

@@ -13,7 +13,11 @@
 // calls (looked up through cudaGetDriverEntryPoint, so the library does not link libcuda), a
 // first-fit free list per slab, and the state machine.  Commit flips every slab to read-only;
 // re-acquiring write access flips it back and keeps contents and addresses (repair in place).
-// What is not here: the separate service process and descriptor passing over Unix sockets.
+// Across processes (Section 4, GMS paragraph: the service keeps the creator handles and hands clients file
+// descriptors over Unix sockets; clients import them, map them and set their own access): a service created
+// with GMS_SERVICE_SHAREABLE makes its slabs exportable, gms_service_export_fd turns a slab into a descriptor,
+// and gms_import_* is the client's side -- import, reserve (at the service's address if asked), map, read-only
+// or writable.  The socket and the messages on it belong to the processes that use this, not to the library.
 // A dry-run backend (no CUDA call, addresses from a counter) lets the bookkeeping be tested without
 // a GPU.  Nothing in this file ever writes through a read-only mapping.
 #include <algorithm>
@@ -38,6 +42,8 @@ struct Driver {
     CUresult (*memSetAccess)(CUdeviceptr, size_t, const CUmemAccessDesc *, size_t) = nullptr;
     CUresult (*memGetAccess)(unsigned long long *, const CUmemLocation *, CUdeviceptr) = nullptr;
     CUresult (*memGetAllocationGranularity)(size_t *, const CUmemAllocationProp *, CUmemAllocationGranularity_flags) = nullptr;
+    CUresult (*memExportToShareableHandle)(void *, CUmemGenericAllocationHandle, CUmemAllocationHandleType, unsigned long long) = nullptr;
+    CUresult (*memImportFromShareableHandle)(CUmemGenericAllocationHandle *, void *, CUmemAllocationHandleType) = nullptr;
     bool ok = false;
 };
 
@@ -63,7 +69,9 @@ Driver *driver()
                lookup("cuMemAddressReserve", &d.memAddressReserve) && lookup("cuMemAddressFree", &d.memAddressFree) &&
                lookup("cuMemMap", &d.memMap) && lookup("cuMemUnmap", &d.memUnmap) && lookup("cuMemSetAccess", &d.memSetAccess) &&
                lookup("cuMemGetAccess", &d.memGetAccess) &&
-               lookup("cuMemGetAllocationGranularity", &d.memGetAllocationGranularity);
+               lookup("cuMemGetAllocationGranularity", &d.memGetAllocationGranularity) &&
+               lookup("cuMemExportToShareableHandle", &d.memExportToShareableHandle) &&
+               lookup("cuMemImportFromShareableHandle", &d.memImportFromShareableHandle);
     });
     return &d;
 }
@@ -88,6 +96,7 @@ struct gms_service {
     std::mutex mu;
     int device = 0;
     bool dry_run = false;
+    bool shareable = false;  // slabs can be exported as file descriptors
     uint64_t slab_bytes = 0, granularity = 2ull << 20;
     uint64_t fake_next_va = 0x700000000000ull;
     uint32_t state = GMS_STATE_EMPTY, readers = 0;
@@ -97,6 +106,16 @@ struct gms_service {
 };
 
 namespace {
+
+CUmemAllocationProp slab_prop(int device, bool shareable)
+{
+    CUmemAllocationProp prop = {};
+    prop.type = CU_MEM_ALLOCATION_TYPE_PINNED;
+    prop.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
+    prop.location.id = device;
+    if (shareable) prop.requestedHandleTypes = CU_MEM_HANDLE_TYPE_POSIX_FILE_DESCRIPTOR;
+    return prop;
+}
 
 int set_access(gms_service *s, const Slab &slab, bool writable)
 {
@@ -118,10 +137,7 @@ int new_slab(gms_service *s, uint64_t size, bool dedicated, Slab *out)
         s->fake_next_va += slab.size + (1ull << 30);
     } else {
         Driver *d = driver();
-        CUmemAllocationProp prop = {};
-        prop.type = CU_MEM_ALLOCATION_TYPE_PINNED;
-        prop.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
-        prop.location.id = s->device;
+        const CUmemAllocationProp prop = slab_prop(s->device, s->shareable);
         CUresult r = d->memCreate(&slab.handle, slab.size, &prop, 0);
         if (r != CUDA_SUCCESS) return r == CUDA_ERROR_OUT_OF_MEMORY ? GMS_ERR_NOMEM : GMS_ERR_CUDA;
         CUdeviceptr va = 0;
@@ -204,10 +220,11 @@ int gms_service_create(uint64_t slab_bytes, uint32_t flags, gms_service **out)
 {
     if (!out) return GMS_ERR_NULL;
     *out = nullptr;
-    if (flags & ~GMS_SERVICE_DRY_RUN) return GMS_ERR_ARG;
+    if (flags & ~(GMS_SERVICE_DRY_RUN | GMS_SERVICE_SHAREABLE)) return GMS_ERR_ARG;
     gms_service *s = new (std::nothrow) gms_service();
     if (!s) return GMS_ERR_NOMEM;
     s->dry_run = (flags & GMS_SERVICE_DRY_RUN) != 0;
+    s->shareable = (flags & GMS_SERVICE_SHAREABLE) != 0;
     if (!s->dry_run) {
         cudaError_t e = cudaFree(nullptr);  // make sure the primary context exists and is current
         if (e == cudaSuccess) e = cudaGetDevice(&s->device);
@@ -219,10 +236,7 @@ int gms_service_create(uint64_t slab_bytes, uint32_t flags, gms_service **out)
             delete s;
             return GMS_ERR_CUDA;
         }
-        CUmemAllocationProp prop = {};
-        prop.type = CU_MEM_ALLOCATION_TYPE_PINNED;
-        prop.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
-        prop.location.id = s->device;
+        const CUmemAllocationProp prop = slab_prop(s->device, s->shareable);
         size_t g = 0;
         if (driver()->memGetAllocationGranularity(&g, &prop, CU_MEM_ALLOC_GRANULARITY_RECOMMENDED) != CUDA_SUCCESS || g == 0) {
             delete s;
@@ -370,10 +384,7 @@ int gms_service_back_pages(gms_service *s)
     if (s->state != GMS_STATE_RW || s->backed) return GMS_ERR_STATE;
     if (!s->dry_run) {
         Driver *d = driver();
-        CUmemAllocationProp prop = {};
-        prop.type = CU_MEM_ALLOCATION_TYPE_PINNED;
-        prop.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
-        prop.location.id = s->device;
+        const CUmemAllocationProp prop = slab_prop(s->device, s->shareable);
         size_t done = 0;
         int rc = GMS_OK;
         for (; done < s->slabs.size() && rc == GMS_OK; ++done) {
@@ -464,6 +475,138 @@ int gms_service_access(gms_service *s, const void *dptr, uint32_t *writable)
         return GMS_OK;
     }
     return GMS_ERR_RANGE;  // not an address of this service
+}
+
+int gms_service_slab(gms_service *s, uint64_t index, gms_slab_info *out)
+{
+    if (!s || !out) return GMS_ERR_NULL;
+    std::lock_guard<std::mutex> l(s->mu);
+    if (index >= s->slabs.size()) return GMS_ERR_RANGE;
+    const Slab &slab = s->slabs[index];
+    gms_slab_info info = {};
+    info.address = slab.va;
+    info.bytes = slab.size;
+    info.dedicated = slab.dedicated ? 1u : 0u;
+    *out = info;
+    return GMS_OK;
+}
+
+int gms_service_export_fd(gms_service *s, uint64_t index, int *fd)
+{
+    if (!s || !fd) return GMS_ERR_NULL;
+    *fd = -1;
+    std::lock_guard<std::mutex> l(s->mu);
+    if (index >= s->slabs.size()) return GMS_ERR_RANGE;
+    if (!s->shareable || s->dry_run || !s->backed) return GMS_ERR_STATE;
+    int h = -1;
+    if (driver()->memExportToShareableHandle(&h, s->slabs[index].handle, CU_MEM_HANDLE_TYPE_POSIX_FILE_DESCRIPTOR, 0) != CUDA_SUCCESS)
+        return GMS_ERR_CUDA;
+    *fd = h;
+    return GMS_OK;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------- the client's side
+struct gms_import {
+    struct Range {
+        uint64_t va = 0, size = 0;
+        CUmemGenericAllocationHandle handle = 0;
+        bool mapped = false;
+    };
+    std::vector<Range> ranges;
+};
+
+extern "C" {
+
+int gms_import_create(const int *fds, const gms_slab_info *slabs, size_t n, uint32_t flags, gms_import **out)
+{
+    if (!out || (n && (!fds || !slabs))) return GMS_ERR_NULL;
+    *out = nullptr;
+    if (flags & ~(GMS_IMPORT_WRITABLE | GMS_IMPORT_SAME_ADDRESS)) return GMS_ERR_ARG;
+    cudaError_t e = cudaFree(nullptr);  // make sure the primary context exists and is current
+    int device = 0;
+    if (e == cudaSuccess) e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return gms::report_cuda_error(e);
+    Driver *d = driver();
+    if (!d->ok) return GMS_ERR_CUDA;
+    gms_import *imp = new (std::nothrow) gms_import();
+    if (!imp) return GMS_ERR_NOMEM;
+    int rc = GMS_OK;
+    try {
+        imp->ranges.reserve(n);
+    } catch (const std::bad_alloc &) {
+        delete imp;
+        return GMS_ERR_NOMEM;
+    }
+    for (size_t i = 0; i < n && rc == GMS_OK; ++i) {
+        gms_import::Range r;
+        r.size = slabs[i].bytes;
+        if (fds[i] < 0 || r.size == 0) {
+            rc = GMS_ERR_ARG;
+            break;
+        }
+        if (d->memImportFromShareableHandle(&r.handle, reinterpret_cast<void *>(static_cast<uintptr_t>(fds[i])),
+                                            CU_MEM_HANDLE_TYPE_POSIX_FILE_DESCRIPTOR) != CUDA_SUCCESS) {
+            rc = GMS_ERR_CUDA;
+            break;
+        }
+        // the service's address is asked for; whether any other one will do is the caller's choice
+        CUdeviceptr va = 0;
+        if (d->memAddressReserve(&va, r.size, 0, (CUdeviceptr)slabs[i].address, 0) != CUDA_SUCCESS) {
+            d->memRelease(r.handle);
+            rc = GMS_ERR_CUDA;
+            break;
+        }
+        r.va = (uint64_t)va;
+        imp->ranges.push_back(r);  // from here on gms_import_destroy undoes it
+        if ((flags & GMS_IMPORT_SAME_ADDRESS) && r.va != slabs[i].address) {
+            rc = GMS_ERR_RANGE;
+            break;
+        }
+        if (d->memMap(va, r.size, 0, r.handle, 0) != CUDA_SUCCESS) {
+            rc = GMS_ERR_CUDA;
+            break;
+        }
+        imp->ranges.back().mapped = true;
+        CUmemAccessDesc desc = {};
+        desc.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
+        desc.location.id = device;
+        desc.flags = (flags & GMS_IMPORT_WRITABLE) ? CU_MEM_ACCESS_FLAGS_PROT_READWRITE : CU_MEM_ACCESS_FLAGS_PROT_READ;
+        if (d->memSetAccess(va, r.size, &desc, 1) != CUDA_SUCCESS) rc = GMS_ERR_CUDA;
+    }
+    if (rc != GMS_OK) {
+        (void)gms_import_destroy(imp);
+        return rc;
+    }
+    *out = imp;
+    return GMS_OK;
+}
+
+int gms_import_address(const gms_import *imp, size_t index, void **dptr)
+{
+    if (!imp || !dptr) return GMS_ERR_NULL;
+    if (index >= imp->ranges.size()) return GMS_ERR_RANGE;
+    *dptr = reinterpret_cast<void *>(imp->ranges[index].va);
+    return GMS_OK;
+}
+
+int gms_import_destroy(gms_import *imp)
+{
+    if (!imp) return GMS_OK;
+    int rc = GMS_OK;
+    if (!imp->ranges.empty()) {
+        cudaError_t e = cudaDeviceSynchronize();  // nothing of this process may still be using the mappings
+        if (e != cudaSuccess) rc = gms::report_cuda_error(e);
+    }
+    Driver *d = driver();
+    for (gms_import::Range &r : imp->ranges) {
+        if (r.mapped && d->memUnmap((CUdeviceptr)r.va, r.size) != CUDA_SUCCESS) rc = GMS_ERR_CUDA;
+        if (r.va && d->memAddressFree((CUdeviceptr)r.va, r.size) != CUDA_SUCCESS) rc = GMS_ERR_CUDA;
+        if (r.handle && d->memRelease(r.handle) != CUDA_SUCCESS) rc = GMS_ERR_CUDA;
+    }
+    delete imp;
+    return rc;
 }
 
 }  // extern "C"

@@ -39,6 +39,7 @@ EXPORTS = (
     "gms_service_create", "gms_service_destroy", "gms_service_acquire_rw", "gms_service_alloc", "gms_service_commit",
     "gms_service_abort", "gms_service_acquire_ro", "gms_service_release_ro", "gms_service_info", "gms_service_access",
     "gms_service_detach", "gms_service_reattach", "gms_service_release_pages", "gms_service_back_pages",
+    "gms_service_slab", "gms_service_export_fd", "gms_import_create", "gms_import_address", "gms_import_destroy",
     "gms_launch_geometry", "gms_kernel_launches", "gms_set_device", "gms_strerror", "gms_last_cuda_error", "gms_version",
 )
 
@@ -119,6 +120,11 @@ def lib():
             "gms_service_reattach": (i, [p]),
             "gms_service_release_pages": (i, [p]),
             "gms_service_back_pages": (i, [p]),
+            "gms_service_slab": (i, [p, u64, p]),
+            "gms_service_export_fd": (i, [p, u64, p]),
+            "gms_import_create": (i, [p, p, C.c_size_t, u32, p]),
+            "gms_import_address": (i, [p, C.c_size_t, p]),
+            "gms_import_destroy": (i, [p]),
             "gms_launch_geometry": (i, [pu32, pu32, pu32]),
             "gms_kernel_launches": (u64, []),
             "gms_set_device": (i, [i]),
@@ -480,3 +486,56 @@ def gms_strerror(status: int) -> str:
 
 def gms_version() -> int:
     return lib().gms_version()
+
+
+# ---------------------------------------------------------------- across processes
+SERVICE_SHAREABLE = 2
+IMPORT_WRITABLE, IMPORT_SAME_ADDRESS = 1, 2
+
+
+class SlabInfo(C.Structure):
+    _fields_ = [("address", C.c_uint64), ("bytes", C.c_uint64), ("dedicated", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+def gms_service_slab(s: Service, index: int) -> dict:
+    info = SlabInfo()
+    _check(lib().gms_service_slab(s.handle, int(index), C.byref(info)), "gms_service_slab")
+    return {"address": info.address, "bytes": info.bytes, "dedicated": info.dedicated}
+
+
+def gms_service_export_fd(s: Service, index: int) -> int:
+    """A new file descriptor for the slab (send it with SCM_RIGHTS, then close it)."""
+    fd = C.c_int(-1)
+    _check(lib().gms_service_export_fd(s.handle, int(index), C.byref(fd)), "gms_service_export_fd")
+    return fd.value
+
+
+class Import:
+    """Owner of a ``gms_import*`` (slabs of another process's service mapped into this one)."""
+
+    def __init__(self, handle, n):
+        self.handle, self.n = handle, n
+
+    def address(self, index: int) -> int:
+        p = C.c_void_p()
+        _check(lib().gms_import_address(self.handle, int(index), C.byref(p)), "gms_import_address")
+        return p.value
+
+    def close(self):
+        if self.handle:
+            lib().gms_import_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+
+def gms_import_create(fds, slabs, flags: int = 0) -> Import:
+    """``slabs``: the dicts of gms_service_slab, in the order of ``fds``."""
+    n = len(fds)
+    cf = (C.c_int * max(n, 1))(*[int(f) for f in fds])
+    cs = (SlabInfo * max(n, 1))()
+    for k, sl in enumerate(slabs):
+        cs[k].address, cs[k].bytes, cs[k].dedicated = int(sl["address"]), int(sl["bytes"]), int(sl.get("dedicated", 0))
+    out = C.c_void_p()
+    _check(lib().gms_import_create(cf, cs, n, flags, C.byref(out)), "gms_import_create")
+    return Import(out.value, n)

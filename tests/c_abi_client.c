@@ -33,6 +33,7 @@ int main(void)
         (fn)gms_service_acquire_rw, (fn)gms_service_alloc, (fn)gms_service_commit, (fn)gms_service_abort,
         (fn)gms_service_acquire_ro, (fn)gms_service_release_ro, (fn)gms_service_info, (fn)gms_service_access,
         (fn)gms_service_detach, (fn)gms_service_reattach, (fn)gms_service_release_pages, (fn)gms_service_back_pages,
+        (fn)gms_service_slab, (fn)gms_service_export_fd, (fn)gms_import_create, (fn)gms_import_address, (fn)gms_import_destroy,
         (fn)gms_launch_geometry, (fn)gms_kernel_launches, (fn)gms_set_device, (fn)gms_strerror, (fn)gms_last_cuda_error,
         (fn)gms_version,
     };
