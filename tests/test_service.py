@@ -286,3 +286,90 @@ def test_addresses_outlive_their_mappings(oracle):
     gms.gms_service_commit(svc)
     m.close()
     svc.close()
+
+
+@pytest.mark.gpu
+def test_kv_pool_owned_by_the_service_is_reattached_and_checked(oracle):
+    """Section 6, "Preserving KV state": for device-preserving failures the service could own the physical KV pages, so that
+    KV contents stay resident and are reattached after recovery.  Here a paged KV pool lives in a slab of its own: filled in
+    state RW (gms_kv_restore), committed, unmapped and mapped again at the same address (detach / reattach), then checked
+    where it lies on the read-only mapping (gms_kv_digest + gms_kv_verify) -- intact; after a writer changed two blocks, the
+    check names them as the oracle does.  Nothing writes through a read-only mapping."""
+    import torch
+
+    n_planes, n_blocks, bb = 6, 96, 32768
+    k = bb // 4096
+    plane_stride = n_blocks * bb
+    pool_bytes = n_planes * plane_stride  # 18 MiB: larger than the slab size, so the pool gets a dedicated slab
+    svc = gms.gms_service_create(8 * MiB)
+    gms.gms_service_acquire_rw(svc)
+    base = gms.gms_service_alloc(svc, pool_bytes)
+    assert gms.gms_service_info(svc)["n_dedicated"] == 1
+    desc = gms.KvPool(base=base, plane_stride=plane_stride, block_stride=bb, n_planes=n_planes, n_blocks=n_blocks, block_bytes=bb)
+    rng = np.random.default_rng(91)
+    everything = rng.permutation(n_blocks).astype(np.int32)
+    image_h = W.random_bytes_host(n_planes * n_blocks * bb, seed=92)
+    pool_h = np.zeros(pool_bytes, np.uint8)
+    rc, _, _, _ = oracle.kv_restore(pool_h, plane_stride, bb, n_planes, n_blocks, bb, image_h, n_blocks * bb, bb, everything)
+    assert rc == 0
+    st = torch.zeros(4, dtype=torch.int64, device="cuda")
+    gms.gms_kv_restore(desc, torch.from_numpy(image_h).cuda(), n_blocks * bb, bb, gms.SRC_DEVICE, torch.from_numpy(everything).cuda(),
+                       n_blocks, None, None, st)
+    torch.cuda.synchronize()
+    assert st[:2].tolist() == [0, 0]
+
+    # the committed blocks an engine would come back to: a third of the pool, in list order
+    ids = rng.permutation(n_blocks)[:32].astype(np.int32)
+    ids_d = torch.from_numpy(ids).cuda()
+    n_slots = len(ids) * n_planes * k
+    recorded = torch.zeros(n_slots, dtype=torch.int64, device="cuda")
+    gms.gms_kv_digest(desc, ids_d, len(ids), recorded, None, st)
+    torch.cuda.synchronize()
+    rc, obd, okd, _ = oracle.kv_digest(pool_h, plane_stride, bb, n_planes, n_blocks, bb, ids)
+    assert rc == 0 and np.array_equal(recorded.cpu().numpy().view(np.uint64), obd)
+
+    def check():
+        """Digest the selected blocks where they lie and compare with the recorded digests."""
+        now = torch.zeros(n_slots, dtype=torch.int64, device="cuda")
+        kd = torch.zeros(len(ids), dtype=torch.int64, device="cuda")
+        out = torch.zeros(2 * 8, dtype=torch.int64, device="cuda")
+        cnt = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+        scratch = torch.zeros(gms.kv_verify_scratch_words(n_slots), dtype=torch.int32, device="cuda")
+        gms.gms_kv_digest(desc, ids_d, len(ids), now, kd, st)
+        gms.gms_kv_verify(desc, ids_d, len(ids), now, recorded, out, 8, cnt, scratch)
+        torch.cuda.synchronize()
+        count = int(cnt.item())
+        recs = out.cpu().numpy().view(np.uint64)[: 2 * min(count, 8)].view(gms.KV_MISMATCH_DTYPE)
+        return now.cpu().numpy().view(np.uint64), kd.cpu().numpy().view(np.uint64), count, \
+            [(int(r["block_id"]), int(r["plane"]), int(r["sub_block"]), int(r["list_pos"])) for r in recs]
+
+    gms.gms_service_commit(svc)
+    assert gms.gms_service_access(svc, base) is False
+    gms.gms_service_detach(svc)    # the engine is gone: nothing is mapped, the pages stay with the service
+    gms.gms_service_reattach(svc)  # the replacement maps them again, read-only, at the same address
+    gms.gms_service_acquire_ro(svc)
+    assert gms.gms_service_access(svc, base) is False
+    now, kd, count, recs = check()
+    assert np.array_equal(now, obd) and np.array_equal(kd, okd) and (count, recs) == (0, [])
+    gms.gms_service_release_ro(svc)
+
+    # a writer replaces two of the selected blocks (and one that is not selected); the next reader is told which
+    gms.gms_service_acquire_rw(svc)
+    unselected = [b for b in range(n_blocks) if b not in set(ids.tolist())]
+    changed = np.array([ids[5], ids[20], unselected[0]], np.int32)
+    patch_h = W.random_bytes_host(n_planes * len(changed) * bb, seed=93)
+    rc, _, _, _ = oracle.kv_restore(pool_h, plane_stride, bb, n_planes, n_blocks, bb, patch_h, len(changed) * bb, bb, changed)
+    assert rc == 0
+    gms.gms_kv_restore(desc, torch.from_numpy(patch_h).cuda(), len(changed) * bb, bb, gms.SRC_DEVICE, torch.from_numpy(changed).cuda(),
+                       len(changed), None, None, st)
+    gms.gms_service_commit(svc)
+    gms.gms_service_acquire_ro(svc)
+    now, kd, count, recs = check()
+    rc, dbd, dkd, _ = oracle.kv_digest(pool_h, plane_stride, bb, n_planes, n_blocks, bb, ids)
+    ocount, orecs = oracle.kv_verify(n_planes, n_blocks, bb, ids, dbd, obd, 8)
+    assert rc == 0 and np.array_equal(now, dbd) and np.array_equal(kd, dkd)
+    assert ocount == 2 * n_planes * k and count == ocount  # every 4 KiB of both blocks, in every plane
+    assert recs == [(int(r["block_id"]), int(r["plane"]), int(r["sub_block"]), int(r["list_pos"])) for r in orecs]
+    assert {r[0] for r in recs} == {int(ids[5])}  # the first eight records all lie in the block that comes first in the list
+    gms.gms_service_release_ro(svc)
+    svc.close()
