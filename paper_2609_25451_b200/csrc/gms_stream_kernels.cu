@@ -275,10 +275,13 @@ struct ListProvider {
     }
 };
 
-// Units are (plane p, selected slot j), plane-major, so that consecutive units read consecutive
-// 32 KiB runs of the packed image.  Units are claimed in order from one counter (kept in the
-// caller's status array), one step ahead like the list provider, so the reads in flight form a
-// compact moving front of the image.
+// Units are (plane p, selected slot j).  The copying calls walk them plane-major, so that consecutive
+// units read (or write) consecutive 32 KiB runs of the packed image.  The digest-only call has no image
+// and walks them slot-major instead: consecutive units then fill consecutive digest slots (the layout
+// is [j][p][block]), whole lines at a time, where plane-major leaves 64-byte pieces 4 KiB apart
+// (measured on the 60 GB pool: 0.855 against 0.870 ms).  Units are claimed in order from one counter
+// (kept in the caller's status array), one step ahead like the list provider, so the reads in flight
+// form a compact moving front of the image.
 struct KvProvider {
     KvArgs a;
     unsigned int *counter;
@@ -291,7 +294,7 @@ struct KvProvider {
     {
         u_next = __shfl_sync(kFull, raw_next, 0);
         if (lane == 0) raw_next = atomicAdd(counter, 1u);
-        if (u_next < total) id_next = __ldg(a.ids + u_next % a.n_sel);
+        if (u_next < total) id_next = __ldg(a.ids + (a.digest_only ? u_next / a.n_planes : u_next % a.n_sel));
     }
     __device__ __forceinline__ void init(uint32_t lane)
     {
@@ -304,7 +307,8 @@ struct KvProvider {
     {
         const uint32_t k = a.block_bytes >> 12;
         while (u_next < total) {
-            const uint32_t p = u_next / a.n_sel, j = u_next % a.n_sel;
+            const uint32_t p = a.digest_only ? u_next % a.n_planes : u_next / a.n_sel;
+            const uint32_t j = a.digest_only ? u_next / a.n_planes : u_next % a.n_sel;
             const int32_t id = id_next;
             step(lane);
             const uint32_t slot0 = (j * a.n_planes + p) * k;  // digest slots are laid out [j][p][block]
