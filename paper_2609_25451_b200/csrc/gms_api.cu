@@ -379,6 +379,7 @@ int manifest_launch_window(const gms_manifest *m, const SrcWindow &w, const void
     a.expected = nullptr;
     a.seg_count = nullptr;
     a.n_segments = 0;
+    a.l2_keep = 0;
     cudaError_t e = launch_restore(a, s);
     return e == cudaSuccess ? GMS_OK : cuda_fail(e);
 }
@@ -673,6 +674,7 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
     a.expected = compare ? m->d_expected : nullptr;
     a.seg_count = compare ? m->d_seg_count : nullptr;
     a.n_segments = compare ? m->n_segments : 0;
+    a.l2_keep = !store && m->n_blocks * sizeof(uint64_t) <= gms::kL2KeepBytes ? 1u : 0u;
     GMS_CUDA(store ? gms::launch_restore(a, static_cast<cudaStream_t>(stream))
                    : gms::launch_digest(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
@@ -853,6 +855,7 @@ static int kv_call(const gms_kv_pool *pool, const void *image, uint64_t img_plan
     a.capture = capture ? 1u : 0u;
     a.digest_only = 0u;
     a.by_id = (pool->flags & GMS_KV_IMAGE_BY_ID) ? 1u : 0u;
+    a.l2_keep = 0u;
     GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
 }
@@ -900,6 +903,7 @@ int gms_kv_digest(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t 
     a.kv_digests = d_kv_digests;
     a.status = reinterpret_cast<unsigned long long *>(d_status);
     a.digest_only = 1u;
+    a.l2_keep = (uint64_t)n_sel * pool->n_planes * k * sizeof(uint64_t) <= gms::kL2KeepBytes ? 1u : 0u;
     GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
 }

@@ -59,7 +59,18 @@ struct StreamArgs {
     const uint64_t *expected;      // fused compare: the recorded block digests (null: no compare)
     uint32_t *seg_count;           // fused compare: per-segment mismatch counters, cleared by the prologue
     uint32_t n_segments;
+    uint32_t l2_keep;              // digest-only kernel: 1 = L2 hints on (see kL2KeepBytes)
 };
+
+// The digest-only kernels write 8 bytes per 4 KiB they read.  When that output is small next to the L2 (126 MB),
+// it pays to keep it there for the length of the kernel and let the payload, which is read once, go first: the
+// bulk loads carry an evict-first hint and the digest stores an evict-last one.  Dirty digest lines that trickle
+// out to DRAM one by one in the middle of a read stream cost far more than their bytes (measured with the output
+// confined to 64 KiB: 2.16 against 2.21 ms on a 16 GB manifest), and with the hints the 12 MB of the 60 GB KV
+// pool's digests stay put (0.861 -> 0.843 ms; mixed manifest, 4 MB: 0.339 -> 0.333 ms).  A 31 MB output measured
+// no better with the hints than without (2.206 / 2.208 ms), and the copying kernels measured slower with them
+// (4.72 -> 4.79 ms), so they are used by the digest-only kernels alone, and only below this output size.
+constexpr uint64_t kL2KeepBytes = 16ull << 20;
 
 struct KvArgs {
     uint8_t *pool_base;
@@ -75,6 +86,7 @@ struct KvArgs {
     uint32_t capture;              // 1: gather pool blocks into the image
     uint32_t digest_only;          // 1: digest the selected pool blocks where they lie (no image, nothing written)
     uint32_t by_id;               // 1: the image is pool-shaped (slot = block id), else packed (slot = list position)
+    uint32_t l2_keep;              // digest-only: 1 = L2 hints on (see kL2KeepBytes)
 };
 
 cudaError_t launch_restore(const StreamArgs &a, cudaStream_t s);

@@ -124,6 +124,30 @@ __device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_
                  "r"(src_smem), "r"(bytes)
                  : "memory");
 }
+// The same load with an L2 eviction policy attached (used by the digest-only kernels, see kL2KeepBytes).
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar, uint64_t policy)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                     dst_smem),
+                 "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar), "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void store_u64_hint(uint64_t *p, uint64_t v, uint64_t policy)
+{
+    asm volatile("st.global.L2::cache_hint.u64 [%0], %1, %2;" ::"l"(p), "l"(v), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read()
@@ -341,7 +365,7 @@ struct KvProvider {
 template <int S, bool kStore, class Provider>
 __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint4 *fifo, uint64_t *bars, uint64_t *block_digests,
                                              uint64_t *accum, unsigned long long *status, const uint64_t *expected,
-                                             uint32_t *seg_count)
+                                             uint32_t *seg_count, bool l2_keep)
 {
     static_assert(S <= (int)kFifo, "the chunk fifo must cover the ring");
     constexpr uint32_t LOOK = S - 1;  // blocks in flight ahead of the one being digested
@@ -360,6 +384,9 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
         }
 
     const uint32_t ring_s = smem_u32(ring), bars_s = smem_u32(bars);
+    // digest-only kernels with a small output: payload loads evict-first, digest stores evict-last (see kL2KeepBytes)
+    const bool keep = !kStore && l2_keep;
+    const uint64_t pol_first = l2_policy_evict_first(), pol_last = l2_policy_evict_last();
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < S; ++s) mbar_init(bars_s + 8u * s, 1u);
@@ -430,7 +457,12 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
             }
             if (lane == 0) {
                 mbar_arrive_expect_tx(bars_s + 8u * s, m16 + stall_extra);
-                if (m16) bulk_load(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s);
+                if (m16) {
+                    if (keep)
+                        bulk_load_hint(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s, pol_first);
+                    else
+                        bulk_load(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s);
+                }
             }
             stall_extra = 0;
             ++it_next;
@@ -486,7 +518,12 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
             uint64_t t = 0;
             if (lane < c_blocks) {
                 const uint64_t raw = ((uint64_t)my_hi << 32) | my_lo, myD = raw ^ (raw >> 31);
-                if (block_digests) block_digests[(uint64_t)c_gblock0 + lane] = myD;
+                if (block_digests) {
+                    if (keep)
+                        store_u64_hint(block_digests + (uint64_t)c_gblock0 + lane, myD, pol_last);
+                    else
+                        block_digests[(uint64_t)c_gblock0 + lane] = myD;
+                }
                 if (expected && want != myD) atomicAdd(seg_count + ((c_gblock0 + lane) >> kVerifySegShift), 1u);
                 t = mix_full32(myD ^ ((uint64_t)(c_tblock0 + lane) * kG));
             }
@@ -553,7 +590,7 @@ __global__ void __launch_bounds__(512, 1) gms_stream_kernel(StreamArgs a)
     // for the grid before it to finish before it touches global memory
     asm volatile("griddepcontrol.launch_dependents;");
     run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.tensor_digests, a.status, a.expected,
-                            a.seg_count);
+                            a.seg_count, a.l2_keep != 0);
 }
 
 template <int S, bool kStore>
@@ -566,7 +603,8 @@ __global__ void __launch_bounds__(512, 1) gms_kv_stream_kernel(KvArgs a)
     prov.counter = reinterpret_cast<unsigned int *>(a.status + 2);
     prov.total = a.n_sel * a.n_planes;
     asm volatile("griddepcontrol.launch_dependents;");
-    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, nullptr, nullptr);
+    run_pipeline<S, kStore>(prov, l.ring, l.fifo, l.bars, a.block_digests, a.kv_digests, a.status + 1, nullptr, nullptr,
+                            a.l2_keep != 0);
 }
 
 // Clears the accumulators the streaming kernels XOR / add into (and, for the fused compare, the per-segment
