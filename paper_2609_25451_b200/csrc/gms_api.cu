@@ -674,7 +674,7 @@ static int stream_call(const gms_manifest *m, const void *image, bool store, uin
     a.expected = compare ? m->d_expected : nullptr;
     a.seg_count = compare ? m->d_seg_count : nullptr;
     a.n_segments = compare ? m->n_segments : 0;
-    a.l2_keep = !store && m->n_blocks * sizeof(uint64_t) <= gms::kL2KeepBytes ? 1u : 0u;
+    a.l2_keep = store ? 0u : gms::l2_keep_for(m->n_blocks);
     GMS_CUDA(store ? gms::launch_restore(a, static_cast<cudaStream_t>(stream))
                    : gms::launch_digest(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
@@ -903,7 +903,7 @@ int gms_kv_digest(const gms_kv_pool *pool, const int32_t *d_block_ids, uint32_t 
     a.kv_digests = d_kv_digests;
     a.status = reinterpret_cast<unsigned long long *>(d_status);
     a.digest_only = 1u;
-    a.l2_keep = (uint64_t)n_sel * pool->n_planes * k * sizeof(uint64_t) <= gms::kL2KeepBytes ? 1u : 0u;
+    a.l2_keep = gms::l2_keep_for((uint64_t)n_sel * pool->n_planes * k);
     GMS_CUDA(gms::launch_kv_restore(a, static_cast<cudaStream_t>(stream)));
     return GMS_OK;
 }

@@ -69,8 +69,15 @@ struct StreamArgs {
 // confined to 64 KiB: 2.16 against 2.21 ms on a 16 GB manifest), and with the hints the 12 MB of the 60 GB KV
 // pool's digests stay put (0.861 -> 0.843 ms; mixed manifest, 4 MB: 0.339 -> 0.333 ms).  A 31 MB output measured
 // no better with the hints than without (2.206 / 2.208 ms), and the copying kernels measured slower with them
-// (4.72 -> 4.79 ms), so they are used by the digest-only kernels alone, and only below this output size.
+// (4.72 -> 4.79 ms), so they are used by the digest-only kernels alone, and only below this output size.  Nor
+// for a payload that the L2 could hold itself: marking it evict-first costs the call that comes next (tiny
+// manifest, 34 MB: the restore behind the digest pass 22.4 -> 23.2 us).
 constexpr uint64_t kL2KeepBytes = 16ull << 20;
+constexpr uint64_t kL2KeepMinBlocks = (256ull << 20) / kBlockBytes;  // payloads from 256 MiB on (twice the L2)
+inline uint32_t l2_keep_for(uint64_t n_blocks)
+{
+    return n_blocks >= kL2KeepMinBlocks && n_blocks * sizeof(uint64_t) <= kL2KeepBytes ? 1u : 0u;
+}
 
 struct KvArgs {
     uint8_t *pool_base;

@@ -135,13 +135,13 @@ __device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void *sr
 __device__ __forceinline__ uint64_t l2_policy_evict_first()
 {
     uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
 __device__ __forceinline__ uint64_t l2_policy_evict_last()
 {
     uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
 __device__ __forceinline__ void store_u64_hint(uint64_t *p, uint64_t v, uint64_t policy)
