@@ -582,6 +582,9 @@ int gms_import_destroy(gms_import *imp);
  *       (defaults 1,1 / 2,1; counters 1..32, chunks 1..64)
  *   GMS_CHUNK_BLOCKS / GMS_CHUNK_BLOCKS_DIGEST         4 KiB blocks per chunk of the copy list and of the digest
  *       list (defaults 4 / 8, fewer for small manifests; 1..32)
+ *   GMS_L2_KEEP                                        0 / 1: never / always give the digest-only kernels their L2
+ *       hints (payload loads evict-first, digest stores evict-last); by default they are used for payloads from
+ *       256 MiB on whose digests take at most 16 MiB
  *   GMS_CHECK_TABLES                                   1: gms_manifest_build reads the work lists it wrote on the
  *       device back and compares them with a host construction of the same lists (GMS_ERR_STATE if they differ)
  */

@@ -221,6 +221,12 @@ int check_kind(const void *image, uint32_t kind)
 }  // namespace
 
 namespace gms {
+uint32_t l2_keep_for(uint64_t n_blocks)
+{
+    static const long forced = env_hook("GMS_L2_KEEP", 0, 1, -1);  // test hook: 0 = never, 1 = always
+    if (forced >= 0) return (uint32_t)forced;
+    return n_blocks >= kL2KeepMinBlocks && n_blocks * sizeof(uint64_t) <= kL2KeepBytes ? 1u : 0u;
+}
 void count_launches(uint32_t n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 int report_cuda_error(cudaError_t e) { return cuda_fail(e); }
 }  // namespace gms

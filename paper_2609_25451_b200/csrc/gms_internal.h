@@ -74,10 +74,7 @@ struct StreamArgs {
 // manifest, 34 MB: the restore behind the digest pass 22.4 -> 23.2 us).
 constexpr uint64_t kL2KeepBytes = 16ull << 20;
 constexpr uint64_t kL2KeepMinBlocks = (256ull << 20) / kBlockBytes;  // payloads from 256 MiB on (twice the L2)
-inline uint32_t l2_keep_for(uint64_t n_blocks)
-{
-    return n_blocks >= kL2KeepMinBlocks && n_blocks * sizeof(uint64_t) <= kL2KeepBytes ? 1u : 0u;
-}
+uint32_t l2_keep_for(uint64_t n_blocks);  // 1 if a digest-only pass over n_blocks blocks gets the hints (hook: GMS_L2_KEEP)
 
 struct KvArgs {
     uint8_t *pool_base;

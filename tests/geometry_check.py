@@ -1,6 +1,6 @@
 """Helper run as a subprocess by test_gpu_shapes.py: the launch shape of the streaming kernels is
 fixed once per process (environment hooks), so every shape needs a process of its own.  Checks
-restore / digest / capture / kv-restore against the oracle on one small odd-sized workload and
+restore / digest / capture / digest + verify in one pass / kv-restore / kv-digest against the oracle on one small odd-sized workload and
 prints OK."""
 import os
 import sys
@@ -38,6 +38,15 @@ def main():
     want = np.full(w.image_bytes, 0x11, np.uint8)
     oracle.capture(rec, want, slab_h)
     assert np.array_equal(back.cpu().numpy(), want) and np.array_equal(payload_of(d.bd, d.nb), obd)
+    # digest + verify in one pass after host-made damage: digests, count and ordered pairs as the oracle has them
+    gms.gms_manifest_set_expected(d.m, torch.from_numpy(obd.view(np.int64)).cuda())
+    for row, byte, bit in W.flip_positions(w, 5, seed=21):
+        d.flip(row, byte, bit)
+    rc, dbd, dtd = oracle.digest(rec, d.slab_host())
+    ocount, omm = oracle.verify(rec, dbd, obd, 3)
+    bd, td, count, pairs = d.fused(3)
+    assert np.array_equal(bd, dbd) and np.array_equal(td, dtd) and count == ocount
+    assert pairs == [(int(r["tensor_id"]), int(r["block"])) for r in omm]
     d.close()
     # kv
     n_planes, n_blocks, bb = 5, 90, 32768
@@ -57,6 +66,13 @@ def main():
     torch.cuda.synchronize()
     assert st[:2].tolist() == [oskip, 0] and np.array_equal(pool.cpu().numpy(), want_pool)
     assert np.array_equal(kb.cpu().numpy().view(np.uint64), okb) and np.array_equal(kd.cpu().numpy().view(np.uint64), okd)
+    # the same blocks digested where they lie
+    rc, dkb, dkd, dskip = oracle.kv_digest(want_pool, n_blocks * bb, bb, n_planes, n_blocks, bb, ids)
+    kb.fill_(-1), kd.fill_(-1)
+    gms.gms_kv_digest(desc, torch.from_numpy(ids).cuda(), len(ids), kb, kd, st)
+    torch.cuda.synchronize()
+    assert st[:2].tolist() == [dskip, 0] and np.array_equal(pool.cpu().numpy(), want_pool)
+    assert np.array_equal(kb.cpu().numpy().view(np.uint64), dkb) and np.array_equal(kd.cpu().numpy().view(np.uint64), dkd)
     print("OK", gms.gms_launch_geometry())
 
 

@@ -27,6 +27,8 @@ SHAPES = [
     {"GMS_GEOM_RESTORE": "6,4,2", "GMS_GEOM_DIGEST": "8,3,2", "GMS_GEOM_KV": "4,6,2", "GMS_CLAIM_RESTORE": "8,3",
      "GMS_CLAIM_DIGEST": "1,1", "GMS_CHUNK_BLOCKS": "7", "GMS_CHUNK_BLOCKS_DIGEST": "2"},
     {"GMS_GEOM_RESTORE": "16,3,1", "GMS_CLAIM_RESTORE": "32,2", "GMS_CLAIM_DIGEST": "32,64", "GMS_CHUNK_BLOCKS_DIGEST": "32"},
+    {"GMS_L2_KEEP": "1"},  # the digest-only kernels' L2 hints, which small cases would not get by themselves
+    {"GMS_L2_KEEP": "1", "GMS_GEOM_DIGEST": "12,4,1", "GMS_CHUNK_BLOCKS_DIGEST": "3"},
 ]
 
 
