@@ -127,9 +127,8 @@ __device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_
 // The same load with an L2 eviction policy attached (used by the digest-only kernels, see kL2KeepBytes).
 __device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar, uint64_t policy)
 {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
-                     dst_smem),
-                 "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar), "l"(policy)
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst_smem), "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(bar), "l"(policy)
                  : "memory");
 }
 __device__ __forceinline__ uint64_t l2_policy_evict_first()
