@@ -71,7 +71,9 @@ struct StreamArgs {
 // no better with the hints than without (2.206 / 2.208 ms), and the copying kernels measured slower with them
 // (4.72 -> 4.79 ms), so they are used by the digest-only kernels alone, and only below this output size.  Nor
 // for a payload that the L2 could hold itself: marking it evict-first costs the call that comes next (tiny
-// manifest, 34 MB: the restore behind the digest pass 22.4 -> 23.2 us).
+// manifest, 34 MB: the restore behind the digest pass 22.4 -> 23.2 us).  The price: after such a call up to
+// 16 MiB of digest lines sit in L2 at the higher retention priority until the cache replaces them (it is a
+// replacement hint, not a reservation: nothing is pinned and nothing has to be reset).
 constexpr uint64_t kL2KeepBytes = 16ull << 20;
 constexpr uint64_t kL2KeepMinBlocks = (256ull << 20) / kBlockBytes;  // payloads from 256 MiB on (twice the L2)
 uint32_t l2_keep_for(uint64_t n_blocks);  // 1 if a digest-only pass over n_blocks blocks gets the hints (hook: GMS_L2_KEEP)
