@@ -414,12 +414,12 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
     uint32_t run_tensor = 0xffffffffu;
     uint64_t run_val = 0;
 
-    for (;;) {
-        // ---------------- issue: keep LOOK blocks ahead
-        while (more && issued - consumed < LOOK) {
+    // ---------------- issue the next block of the work list (false: the list is exhausted)
+    auto issue_one = [&]() -> bool {
+        {
             if (it_next == it_blocks) {
                 more = prov.next(it, lane);
-                if (!more) break;
+                if (!more) return false;
                 it_blocks = (it.nbytes + kBlockBytes - 1) >> 12;
                 it_full = it.nbytes >> 12;  // whole blocks: nothing to pad, no hand-moved tail
                 stall_extra = it.stall;     // self-test only: announced on the chunk's first barrier, never sent
@@ -467,8 +467,13 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
             ++it_next;
             ++issued;
         }
-        if (consumed == issued) break;
-
+        return true;
+    };
+    // LOOK blocks go out first; after that every digested block is followed by one more issue, so the warp always
+    // has LOOK blocks in flight or in work
+    for (uint32_t k = 0; k < LOOK; ++k)
+        if (!issue_one()) break;
+    while (consumed != issued) {
         // ---------------- digest block `consumed`
         const uint32_t s = cs;
         const bool ok = mbar_wait_bounded(bars_s + 8u * s, cparity);
@@ -537,6 +542,7 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
         }
         __syncwarp();  // every lane is done reading the slot before it is refilled
         ++consumed;
+        if (more) issue_one();
     }
 
     if (run_tensor != 0xffffffffu && lane == 0 && accum)
