@@ -105,12 +105,6 @@ __device__ __forceinline__ bool mbar_wait_until(uint32_t bar, uint32_t parity, u
     }
     return false;
 }
-// Wait for a phase of one of the warp's own barriers; false after kWaitLimitNs.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_until(bar, parity, global_timer_ns() + kWaitLimitNs);
-}
 // 1-D bulk copy global -> shared (bytes: multiple of 16, both addresses 16-byte aligned).
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
 {
@@ -488,10 +482,14 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
     auto step = [&](auto slot_c) -> bool {
         constexpr uint32_t s = decltype(slot_c)::value;
         if (consumed == issued) return false;
-        const bool ok = mbar_wait_bounded(bars_s + 8u * s, parity);
-        if (!__all_sync(kFull, ok)) {
-            failed = true;
-            return false;
+        // one poll by every lane and a vote on it: the common case costs no divergent branch; only when some lane has
+        // not seen the block yet does the warp go into the bounded wait together
+        if (!__all_sync(kFull, mbar_try_wait(bars_s + 8u * s, parity))) {
+            const bool ok = mbar_wait_until(bars_s + 8u * s, parity, global_timer_ns() + kWaitLimitNs);
+            if (!__all_sync(kFull, ok)) {
+                failed = true;
+                return false;
+            }
         }
         __syncwarp();
         if (c_next == c_blocks) {  // next chunk record
