@@ -42,7 +42,6 @@
 // it has in flight and returns.
 #include <algorithm>
 #include <mutex>
-#include <type_traits>
 
 #include "gms_internal.h"
 
@@ -104,6 +103,12 @@ __device__ __forceinline__ bool mbar_wait_until(uint32_t bar, uint32_t parity, u
         if (global_timer_ns() > deadline) return false;
     }
     return false;
+}
+// Wait for a phase of one of the warp's own barriers; false after kWaitLimitNs.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_until(bar, parity, global_timer_ns() + kWaitLimitNs);
 }
 // 1-D bulk copy global -> shared (bytes: multiple of 16, both addresses 16-byte aligned).
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
@@ -352,37 +357,6 @@ struct KvProvider {
 };
 
 // ---------------------------------------------------------------- the per-warp pipeline
-// Calls f(integral_constant<int, I>) for I = 0 .. N-1 in order until one of them returns false.
-template <int I, int N, class F>
-__device__ __forceinline__ bool static_all(F &f)
-{
-    if constexpr (I < N) {
-        if (!f(std::integral_constant<int, I>{})) return false;
-        return static_all<I + 1, N>(f);
-    } else {
-        return true;
-    }
-}
-// Short last block of a tensor (m < 4096 bytes of it exist): zero-fills the ring slot past the part a bulk copy can
-// move and moves the last m % 16 bytes by hand (into the slot and, when copying, to the destination).  Returns the
-// size of the bulk part.  Kept out of line: it runs once per tensor at most and would otherwise be repeated in
-// every unrolled step of the pipeline.
-template <bool kStore>
-__device__ __noinline__ uint32_t stage_short_block(uint8_t *stage, const uint8_t *src, uint8_t *dst, uint32_t m, uint32_t lane)
-{
-    const uint32_t m16 = m & ~15u;
-    __syncwarp();
-    for (uint32_t o = m16 + 16u * lane; o < kBlockBytes; o += 512u) *reinterpret_cast<uint4 *>(stage + o) = make_uint4(0, 0, 0, 0);
-    __syncwarp();
-    if (lane < (m & 15u)) {
-        const uint8_t v = src[m16 + lane];
-        stage[m16 + lane] = v;
-        if (kStore) dst[m16 + lane] = v;
-    }
-    fence_proxy_async_smem();  // generic writes to a slot that bulk copies will overwrite later
-    __syncwarp();
-    return m16;
-}
 // `expected` / `seg_count` (both null, or both set): the fused compare.  At the end of a chunk every lane that holds
 // a block digest checks it against the recorded one and, if they differ, bumps the counter of the 2048-slot
 // segment the block lies in -- the first pass of the ordered compaction in gms_verify_kernels.cu, done here
@@ -432,64 +406,81 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
     uint32_t c_nbytes = 0, c_tensor = 0, c_gblock0 = 0, c_tblock0 = 0, c_blocks = 0, c_next = 0, chunks_out = 0;
     bool more = true, failed = false;
     uint32_t issued = 0, consumed = 0;
-    uint32_t parity = 0;  // barrier phase of the round (S blocks) being digested
+    uint32_t is = 0;               // ring slot of the next block to issue   (issued % S)
+    uint32_t cs = 0, cparity = 0;  // ring slot and barrier phase of the next block to digest
     uint32_t my_lo = 0, my_hi = 0;
     uint64_t want = 0;  // fused compare: the recorded digest of the block whose digest this lane holds
     // share of a tensor digest gathered over consecutive chunks of the same tensor: one atomic per run, not per chunk
     uint32_t run_tensor = 0xffffffffu;
     uint64_t run_val = 0;
 
-    // The loop below is unrolled over the ring: block k always lives in slot k % S, so every step knows its slot,
-    // its barrier and the slot it refills as constants.
-    // ---------------- issue the next block of the work list into slot `s` (false: the list is exhausted)
-    auto issue_one = [&](auto slot_c) -> bool {
-        constexpr uint32_t s = decltype(slot_c)::value;
-        if (it_next == it_blocks) {
-            more = prov.next(it, lane);
-            if (!more) return false;
-            it_blocks = (it.nbytes + kBlockBytes - 1) >> 12;
-            it_full = it.nbytes >> 12;  // whole blocks: nothing to pad, no hand-moved tail
-            stall_extra = it.stall;     // self-test only: announced on the chunk's first barrier, never sent
-            it_next = 0;
+    // ---------------- issue the next block of the work list (false: the list is exhausted)
+    auto issue_one = [&]() -> bool {
+        {
+            if (it_next == it_blocks) {
+                more = prov.next(it, lane);
+                if (!more) return false;
+                it_blocks = (it.nbytes + kBlockBytes - 1) >> 12;
+                it_full = it.nbytes >> 12;  // whole blocks: nothing to pad, no hand-moved tail
+                stall_extra = it.stall;     // self-test only: announced on the chunk's first barrier, never sent
+                it_next = 0;
+                if (lane == 0) {
+                    const uint64_t d = reinterpret_cast<uint64_t>(it.dst);
+                    fifo[2 * (chunks_in % kFifo)] = make_uint4((uint32_t)d, (uint32_t)(d >> 32), it.nbytes, it.tensor);
+                    fifo[2 * (chunks_in % kFifo) + 1] = make_uint4(it.gblock0, it.tblock0, 0u, 0u);
+                }
+                ++chunks_in;
+            }
+            const uint32_t s = is;
+            is = (is + 1 == S) ? 0 : is + 1;
+            const uint32_t off = it_next << 12;
+            // the slot was last read by the store of block issued-S: all but the newest group must have read
+            if (kStore && lane == 0) bulk_wait_read<S - LOOK>();
+            uint32_t m16 = kBlockBytes;
+            if (it_next >= it_full) {
+                // short last block of a tensor: zero-fill the slot past the bulk part and move the <16 B tail by hand
+                const uint32_t m = it.nbytes - off;
+                m16 = m & ~15u;
+                uint8_t *stage = ring + s * kBlockBytes;
+                __syncwarp();
+                for (uint32_t o = m16 + 16u * lane; o < kBlockBytes; o += 512u)
+                    *reinterpret_cast<uint4 *>(stage + o) = make_uint4(0, 0, 0, 0);
+                __syncwarp();
+                if (lane < (m & 15u)) {
+                    const uint8_t v = it.src[off + m16 + lane];
+                    stage[m16 + lane] = v;
+                    if (kStore) it.dst[off + m16 + lane] = v;
+                }
+                fence_proxy_async_smem();  // generic writes to a slot that bulk copies will overwrite later
+                __syncwarp();
+            }
             if (lane == 0) {
-                const uint64_t d = reinterpret_cast<uint64_t>(it.dst);
-                fifo[2 * (chunks_in % kFifo)] = make_uint4((uint32_t)d, (uint32_t)(d >> 32), it.nbytes, it.tensor);
-                fifo[2 * (chunks_in % kFifo) + 1] = make_uint4(it.gblock0, it.tblock0, 0u, 0u);
+                mbar_arrive_expect_tx(bars_s + 8u * s, m16 + stall_extra);
+                if (m16) {
+                    if (keep)
+                        bulk_load_hint(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s, pol_first);
+                    else
+                        bulk_load(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s);
+                }
             }
-            ++chunks_in;
+            stall_extra = 0;
+            ++it_next;
+            ++issued;
         }
-        const uint32_t off = it_next << 12;
-        // the slot was last read by the store of block issued-S: all but the newest group must have read
-        if (kStore && lane == 0) bulk_wait_read<S - LOOK>();
-        uint32_t m16 = kBlockBytes;
-        if (it_next >= it_full)
-            m16 = stage_short_block<kStore>(ring + s * kBlockBytes, it.src + off, kStore ? it.dst + off : nullptr, it.nbytes - off, lane);
-        if (lane == 0) {
-            mbar_arrive_expect_tx(bars_s + 8u * s, m16 + stall_extra);
-            if (m16) {
-                if (keep)
-                    bulk_load_hint(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s, pol_first);
-                else
-                    bulk_load(ring_s + s * kBlockBytes, it.src + off, m16, bars_s + 8u * s);
-            }
-        }
-        stall_extra = 0;
-        ++it_next;
-        ++issued;
         return true;
     };
-    // ---------------- digest the block in slot `s`, then refill the slot of the block before it
-    auto step = [&](auto slot_c) -> bool {
-        constexpr uint32_t s = decltype(slot_c)::value;
-        if (consumed == issued) return false;
-        // one poll by every lane and a vote on it: the common case costs no divergent branch; only when some lane has
-        // not seen the block yet does the warp go into the bounded wait together
-        if (!__all_sync(kFull, mbar_try_wait(bars_s + 8u * s, parity))) {
-            const bool ok = mbar_wait_until(bars_s + 8u * s, parity, global_timer_ns() + kWaitLimitNs);
-            if (!__all_sync(kFull, ok)) {
-                failed = true;
-                return false;
-            }
+    // LOOK blocks go out first; after that every digested block is followed by one more issue, so the warp always
+    // has LOOK blocks in flight or in work
+    for (uint32_t k = 0; k < LOOK; ++k)
+        if (!issue_one()) break;
+    while (consumed != issued) {
+        // ---------------- digest block `consumed`
+        const uint32_t s = cs;
+        const bool ok = mbar_wait_bounded(bars_s + 8u * s, cparity);
+        if (++cs == S) cs = 0, cparity ^= 1u;
+        if (!__all_sync(kFull, ok)) {
+            failed = true;
+            break;
         }
         __syncwarp();
         if (c_next == c_blocks) {  // next chunk record
@@ -551,14 +542,8 @@ __device__ __forceinline__ void run_pipeline(Provider &prov, uint8_t *ring, uint
         }
         __syncwarp();  // every lane is done reading the slot before it is refilled
         ++consumed;
-        // block `consumed + LOOK - 1` goes into the slot of the block digested before this one
-        if (more) issue_one(std::integral_constant<int, (s + LOOK) % S>{});
-        return true;
-    };
-    // LOOK blocks go out first (slots 0 .. LOOK-1); after that every digested block is followed by one more issue,
-    // so the warp always has LOOK blocks in flight or in work
-    static_all<0, (int)LOOK>(issue_one);
-    while (static_all<0, S>(step)) parity ^= 1u;
+        if (more) issue_one();
+    }
 
     if (run_tensor != 0xffffffffu && lane == 0 && accum)
         atomicXor(reinterpret_cast<unsigned long long *>(accum + run_tensor), (unsigned long long)run_val);
