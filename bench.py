@@ -73,6 +73,7 @@ def parse_args():
                     help="8b/mixed/tiny: capture the step into a CUDA graph once and time its replays (whole step only)")
     ap.add_argument("--no-l2-flush", action="store_true", help="mixed/tiny: leave L2 as the previous step left it")
     ap.add_argument("--file-dir", default="/dev/shm", help="file: where the snapshot file is written")
+    ap.add_argument("--no-file", action="store_true", help="default run: leave the storage-fed entry out")
     ap.add_argument("--pipe-buffers", type=int, default=4)
     ap.add_argument("--pipe-mib", type=int, default=256)
     ap.add_argument("--pipe-readers", type=int, default=16)
@@ -1064,7 +1065,7 @@ def run_host70b(args, torch, gms, W, dev, index, want_cpu=True, cpu_seconds=4.0)
         gms.gms_host_image_free(hptr)
 
 
-def run_file(args, torch, gms, W, dev, index, want_cpu=True):
+def run_file(args, torch, gms, W, dev, index, want_cpu=True, steps_cap=5):
     """Storage-fed restore of the 8B manifest: file -> ring of pinned buffers -> device (gms_restore_fd),
     against (a) the same reader pool filling one pinned buffer with nothing consuming it and (b) the host link."""
     import concurrent.futures as cf
@@ -1113,7 +1114,7 @@ def run_file(args, torch, gms, W, dev, index, want_cpu=True):
         pipe = gms.gms_pipe_create(n_buf, buf_bytes, n_readers)
         gms.gms_pipe_direct_io(pipe, args.direct_io)
         gms.gms_restore_fd(bench.m, pipe, fd, 0, bench.bd, bench.td)
-        steps = max(1, min(args.steps, 5))
+        steps = max(1, min(args.steps, steps_cap))
         sampler = ClockSampler(index)
         launches0 = gms.gms_kernel_launches()
         sampler.start()
@@ -1453,12 +1454,32 @@ def main():
             release(torch)
         line["configs"] = {name: configs[name] for name in CONFIG_ORDER}
         line["config"]["all_five"] = {name: (compact(c) if "error" not in c else c) for name, c in line["configs"].items()}
+        # ---- the storage-fed legs (file -> pinned ring -> copy engine -> device, and back), a sixth entry beside the five
+        if not args.no_file:
+            try:
+                import shutil
+
+                need = W.llama3_8b_manifest().image_bytes + (1 << 30)
+                if shutil.disk_usage(args.file_dir).free < need:
+                    raise RuntimeError(f"{args.file_dir} has less than {need} bytes free")
+                f = run_file(args, torch, gms, W, dev, local_rank, want_cpu=False, steps_cap=2)
+                keep = ("value", "unit", "steps", "ms_per_step", "roofline", "pipe_stats_best", "parity_ok", "capture_fd", "capture_fd_mapped")
+                line["storage_fed"] = {k: f[k] for k in keep if k in f}
+                line["storage_fed"]["workload"] = f["config"]["workload"]
+                line["storage_fed"]["file_system"] = f["config"]["file_system"]
+            except Exception as ex:  # noqa: BLE001  (no room for the file, say: the line stands without this entry)
+                line["storage_fed"] = {"error": f"{type(ex).__name__}: {ex}"[:400], "parity_ok": False}
+            release(torch)
         # last key of the line, so that it survives a reader that keeps only the end of the output
         line["five_configs"] = "; ".join(
             (f"{n}: {c['ms']} ms {c['gbs']} GB/s frac {c['frac']} ({c['bound']}) parity {'ok' if c['parity_ok'] else 'FAILED'}"
              + (f" cpu {c['cpu_gbs']} GB/s x{c['cpu_cores']}" if "cpu_gbs" in c else "")
              + (f", {c['cpu_all_gbs']} x{c['cpu_all_cores']}" if "cpu_all_gbs" in c else "")) if "error" not in c else f"{n}: {c['error'][:80]}"
             for n, c in line["config"]["all_five"].items())
+        sf = line.get("storage_fed")
+        if sf and "error" not in sf:
+            line["five_configs"] += (f"; file-fed restore ({sf['file_system']}): {round(sf['value'], 1)} GB/s frac {round(sf['roofline']['frac'], 3)} "
+                                     f"({sf['roofline']['bound']}) parity {'ok' if sf['parity_ok'] else 'FAILED'}")
     else:
         bench.close()
 
