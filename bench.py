@@ -1454,6 +1454,33 @@ def main():
             release(torch)
         line["configs"] = {name: configs[name] for name in CONFIG_ORDER}
         line["config"]["all_five"] = {name: (compact(c) if "error" not in c else c) for name, c in line["configs"].items()}
+        # ---- the inverse path and the service substrate on the 8B manifest: gms_capture into a device image and into a
+        # pinned host image, and the headline step with the destinations in gms_service VMM slabs
+        extra_steps = max(3, min(args.steps, 10))
+        try:
+            cb = CaptureBench(torch, gms, W, dev)
+            ce = measure(torch, gms, cb, extra_steps, args.warmup, local_rank)
+            line["capture"] = compact(ce)
+            if not args.no_e2e:
+                try:
+                    line["capture"]["to_host"] = capture_to_host_leg(torch, gms, cb)
+                except gms.GmsError as ex:
+                    line["capture"]["to_host"] = {"error": str(ex)[:300]}
+            cb.close()
+            del cb
+        except Exception as ex:  # noqa: BLE001
+            line["capture"] = {"error": f"{type(ex).__name__}: {ex}"[:400], "parity_ok": False}
+        release(torch)
+        try:
+            vb = ManifestBench("8b", torch, gms, W, dev, vmm=True)
+            ve = measure(torch, gms, vb, extra_steps, args.warmup, local_rank)
+            line["vmm_slabs"] = compact(ve)
+            line["vmm_slabs"]["destinations"] = vb.config()["destinations"]
+            vb.close()
+            del vb
+        except Exception as ex:  # noqa: BLE001
+            line["vmm_slabs"] = {"error": f"{type(ex).__name__}: {ex}"[:400], "parity_ok": False}
+        release(torch)
         # ---- the storage-fed legs (file -> pinned ring -> copy engine -> device, and back), a sixth entry beside the five
         if not args.no_file:
             try:
